@@ -1,0 +1,454 @@
+#!/usr/bin/env python
+"""Benchmark of the per-rank MoE expert block on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3-uniform|...] [--impl reference]
+    python bench.py --sweep            # cost-profile sweep (G, N grid) + max-affine fit -> n*
+
+One "step" is one pass of the whole hot path (count+dispatch, permute+quantise, gate/up GEMM + SwiGLU,
+down GEMM, combine) over one seeded synthetic routed batch, replayed as one CUDA graph.  Weight copies
+rotate through a pool larger than L2 so no step finds its weights cached (the paper's calibration
+protocol, Appendix B).  Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "moe_expert_block_us"          # step time / activated expert instances (lower is better)
+UNIT = "us_per_expert_block"
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_FP8_OVER_BF16 = 2.0             # dense fp8 peak = 2 x dense bf16 peak on this part
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the gate/up GEMM from the committed ncu
+# capture (profiles/), keyed by workload; None until a capture exists for that workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def make_workload(name: str, rank: int = 0):
+    from paper_2608_13057_b200 import workloads as W
+    if name == "cfg1":
+        return W.config1(seed=0 + 101 * rank)
+    if name == "cfg2":
+        return W.config2(seed=1 + 101 * rank)
+    if name.startswith("cfg3-"):
+        return W.config3(name[5:].replace("-", "_"), seed=2 + 101 * rank)
+    if name == "cfg4":
+        return W.config4(seed=3 + 101 * rank)
+    if name.startswith("cfg5-"):                       # cfg5-G-N
+        _, G, N = name.split("-")
+        return W.config5_point(int(G), int(N))
+    raise ValueError(name)
+
+
+def workload_stats(wl):
+    """Units of one step, from the routing and the quota table alone (host tally, not timed)."""
+    live = wl.topk_ids[:wl.n_valid].reshape(-1)
+    counts = np.bincount(live[(live >= 0) & (live < wl.E)], minlength=wl.E)
+    rows = []
+    for e in range(wl.E):
+        for r in range(wl.R_max):
+            if wl.replica_map[e, r] >= 0:
+                rows.append(int(wl.quota[e, r]))
+    rows = [m for m in rows if m > 0]
+    tiles = sum(-(-m // 128) for m in rows)
+    return dict(G_act=len(rows), N_local=sum(rows), tiles=tiles, M_pad=128 * tiles,
+                weight_bytes=len(rows) * 3 * wl.d * wl.f, padded_flops=128 * tiles * 6 * wl.d * wl.f,
+                n_valid=int(wl.n_valid), counts_total=int(counts.sum()))
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled in the background while the GPU is timed."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(gpu_index), "-lms", "100"], stdout=self.file,
+                                         stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.file:
+            c = [v.strip() for v in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1]))
+                mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        busy = [v for v in sm if v >= 0.5 * max(sm)] or sm
+        return dict(sm_mhz=float(np.median(busy)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+
+
+# --------------------------------------------------------------------------------------------------
+# CPU oracle legs (the only places bench.py touches oracle/)
+# --------------------------------------------------------------------------------------------------
+
+def oracle_sample_us_per_block(wl, budget_s: float = 15.0):
+    """Times the oracle as it stands on a bounded sample: all of steps 1-2, the FFN of the first few
+    activated instances (until budget_s), extrapolated over instances; plus the combine."""
+    from oracle import tempo_oracle as O
+    t0 = time.perf_counter()
+    disp = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, wl.M_cap)
+    a_q, a_s = O.permute_pad(wl.x, disp["row_pair"], disp["m_pad"], wl.k)
+    t_head = time.perf_counter() - t0
+    act = [i for i in range(wl.G_max) if disp["inst_count"][i] > 0]
+    done, rows_done, t_ffn = 0, 0, 0.0
+    y = np.zeros((len(disp["row_pair"]), wl.d), np.float32)
+    for i in act:
+        lo, hi = int(disp["inst_off"][i]), int(disp["inst_off"][i + 1])
+        w = wl.expert_weights(int(wl.slot_expert[i]))
+        t1 = time.perf_counter()
+        _, _, y[lo:hi] = O.expert_ffn(a_q[lo:hi], a_s[lo:hi], w.w13_q, w.w13_s, w.w2_q, w.w2_s)
+        t_ffn += time.perf_counter() - t1
+        done += 1
+        rows_done += hi - lo
+        if t_ffn > budget_s and done >= 2:
+            break
+    t2 = time.perf_counter()
+    O.combine(y, disp["pair_row"], wl.topk_w, min(wl.n_valid, 256), wl.T, wl.k)
+    t_comb = (time.perf_counter() - t2) * max(1.0, wl.n_valid / 256.0)
+    total = t_head + t_ffn * (len(act) / max(done, 1)) + t_comb
+    sample = (f"steps 1-2 in full, FFN of {done} of {len(act)} activated instances ({rows_done} padded rows) "
+              f"scaled by instance count, combine of {min(wl.n_valid, 256)} rows scaled by rows")
+    return total * 1e6 / max(len(act), 1), sample
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, timed on the host cores, same metric and workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = make_workload(args.workload, 0)
+    wl.slot_weights()
+    st = workload_stats(wl)
+    for _ in range(max(0, min(args.warmup, 1))):
+        oracle_sample_us_per_block(wl, budget_s=2.0)
+    vals, sample = [], ""
+    for _ in range(max(1, min(args.steps, 3))):
+        v, sample = oracle_sample_us_per_block(wl, budget_s=8.0)
+        vals.append(v)
+    v = float(np.mean(vals))
+    cores = os.cpu_count()
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": len(vals),
+        "warmup": min(args.warmup, 1), "ms_per_step": v * st["G_act"] / 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "G_act": st["G_act"], "N_local": st["N_local"]},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# --------------------------------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------------------------------
+
+def _capture_graphs(torch, buf, pools):
+    graphs = []
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for blob in pools:
+            buf.run_block(packed=blob)                  # warm the launch path outside capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    for blob in pools:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            buf.run_block(packed=blob)
+        graphs.append(g)
+    return graphs
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_13057_b200 import binding as B
+    from paper_2608_13057_b200.ranks import reduce_step
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    wl = make_workload(args.workload, rank)
+    st = workload_stats(wl)
+    buf = B.RankBuffers.for_workload(wl)
+    weight_bytes_all = buf.packed.numel()
+    n_pools = max(2, math.ceil((1 << 30) / max(weight_bytes_all, 1)))
+    n_pools = min(n_pools, 64)
+    pools = [buf.packed] + [buf.packed.clone() for _ in range(n_pools - 1)]
+    graphs = _capture_graphs(torch, buf, pools)
+    K, Wm = args.steps, args.warmup
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+
+    # ---- region A: the whole block as one graph replay per step, inputs resident in HBM ------------
+    for i in range(Wm):
+        graphs[i % n_pools].replay()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(K):
+        graphs[i % n_pools].replay()
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    status = int(buf.status.item())
+
+    # ---- region B: the same steps launched call by call with events between the kernels -----------
+    Kb = min(K, 200)
+    names = ["count_dispatch", "permute_pad", "ffn_gate_up", "ffn_down", "unpermute_combine"]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(Kb)]
+    s = buf.shape
+    torch.cuda._sleep(int(4e7))                        # keep the GPU busy so every launch is queued ahead
+    for i in range(Kb):
+        blob = pools[i % n_pools]
+        ev[i][0].record()
+        B.tempo_count_dispatch(s, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts, buf.counts,
+                               buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair, buf.tile_inst, buf.m_pad,
+                               buf.status)
+        ev[i][1].record()
+        B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status)
+        ev[i][2].record()
+        B.tempo_ffn_gate_up(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.status)
+        ev[i][3].record()
+        B.tempo_ffn_down(s, buf.h_q, buf.h_sf, blob, buf.inst_off, buf.m_pad, buf.y, buf.status)
+        ev[i][4].record()
+        B.tempo_unpermute_combine(s, buf.y, buf.pair_row, buf.topk_w, buf.n_valid, buf.out, buf.status)
+        ev[i][5].record()
+    torch.cuda.synchronize()
+    kern_us = {n: float(np.mean([ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(Kb)])) * 1e3
+               for j, n in enumerate(names)}
+
+    # ---- e2e: host buffers in, host result out, every step ------------------------------------------
+    h_ids = torch.from_numpy(wl.topk_ids).pin_memory()
+    h_w = torch.from_numpy(wl.topk_w).pin_memory()
+    h_x = torch.from_numpy(wl.x).to(torch.bfloat16).pin_memory()
+    h_out = torch.empty(wl.T, wl.d, dtype=torch.bfloat16).pin_memory()
+    h2d = h_ids.numel() * 4 + h_w.numel() * 4 + h_x.numel() * 2
+    d2h = h_out.numel() * 2
+
+    def e2e_step(i):
+        buf.topk_ids.copy_(h_ids, non_blocking=True)
+        buf.topk_w.copy_(h_w, non_blocking=True)
+        buf.x.copy_(h_x, non_blocking=True)
+        graphs[i % n_pools].replay()
+        h_out.copy_(buf.out, non_blocking=True)
+
+    Ke = min(K, 500)
+    for i in range(min(Wm, 5)):
+        e2e_step(i)
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for i in range(Ke):
+        e2e_step(i)
+    f1.record()
+    barrier()
+    ms_e2e = f0.elapsed_time(f1) / Ke
+
+    clocks = sampler.stop() if sampler is not None else None
+
+    ms_step, units = reduce_step(ms_total / K, float(st["G_act"]), "cuda" if world > 1 else None)
+    ms_e2e_max, _ = reduce_step(ms_e2e, float(st["G_act"]), "cuda" if world > 1 else None)
+    if world > 1:
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+
+    peaks = _peaks()
+    us_step = ms_step * 1e3
+    hbm_time = st["weight_bytes"] / (peaks["hbm_gbs"] * 1e9) * 1e6
+    fp8_peak = peaks["bf16_tflops_sustained"] * NOMINAL_FP8_OVER_BF16
+    tensor_time = st["padded_flops"] / (fp8_peak * 1e12) * 1e6
+    bound = "hbm" if hbm_time >= tensor_time else "tensor"
+    # dominant kernel: the gate/up GEMM (2/3 of the weight bytes and of the FLOPs)
+    g1_us = kern_us["ffn_gate_up"]
+    if bound == "hbm":
+        alg = st["G_act"] * 2 * wl.d * wl.f                        # bytes: W13 of every activated instance
+        achieved = alg / (g1_us * 1e-6) / 1e9
+        roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=achieved / peaks["hbm_gbs"], traffic=NCU_TRAFFIC_BYTES.get(args.workload))
+    else:
+        alg = st["M_pad"] * 4 * wl.d * wl.f                        # flops: 2 * M_pad * 2f * d
+        achieved = alg / (g1_us * 1e-6) / 1e12
+        roof = dict(bound="tensor", achieved=achieved, peak=fp8_peak, unit="TFLOP/s", frac=achieved / fp8_peak,
+                    traffic=NCU_TRAFFIC_BYTES.get(args.workload))
+    roof.update(kernel="ffn_gemm_kernel<0> (gate/up + SwiGLU)", kernel_us=g1_us, peak_source=peaks["source"] +
+                (" HBM copy" if bound == "hbm" else " bf16 sustained x 2 (nominal fp8/bf16 ratio)"))
+
+    out = {
+        "metric": METRIC, "value": us_step / units, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "T": wl.T, "top_k": wl.k, "E": wl.E, "d": wl.d, "f": wl.f,
+                   "G_act": st["G_act"], "N_local": st["N_local"], "M_pad": st["M_pad"],
+                   "l2": f"weights rotate through {n_pools} copies ({n_pools * weight_bytes_all / 1e9:.2f} GB >> L2)",
+                   "parallelism": f"{world} independent rank(s), no collective"},
+        "block_us": us_step, "tokens_per_s": st["n_valid"] * world / (us_step * 1e-6),
+        "block_roofline": {"weight_us": hbm_time, "padded_flop_us": tensor_time,
+                           "frac": max(hbm_time, tensor_time) / us_step,
+                           "ffn_frac": max(hbm_time, tensor_time) / (kern_us["ffn_gate_up"] + kern_us["ffn_down"])},
+        "kernel_us": kern_us, "gpu_launches": 5 * K, "device_status": status,
+        "roofline": roof, "clocks": clocks,
+        "e2e": {"value": ms_e2e_max * 1e3 / units, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        v, sample = oracle_sample_us_per_block(wl, budget_s=12.0)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "sample": sample}
+    print(json.dumps(out))
+
+
+# --------------------------------------------------------------------------------------------------
+# cost-profile sweep (config 5) and fit
+# --------------------------------------------------------------------------------------------------
+
+def run_sweep(args):
+    import torch
+    from paper_2608_13057_b200 import binding as B
+    from paper_2608_13057_b200 import costmodel as C
+    from paper_2608_13057_b200 import workloads as W
+
+    torch.cuda.set_device(0)
+    d, f = 4096, 1536
+    Gs = [int(g) for g in args.sweep_G.split(",")] if args.sweep_G else list(W.SWEEP_G)
+    Ns = [int(n) for n in args.sweep_N.split(",")] if args.sweep_N else list(W.SWEEP_N)
+    replays = args.replays
+    rows = []
+    gen = torch.Generator(device="cuda").manual_seed(4)
+    for G in Gs:
+        # one weight set per G, copied into a rotation pool >> L2
+        wl0 = W.config5_point(G, 1, with_x=False)
+        probe = B.RankBuffers(G, 1, G, G, 1, d, f)
+        packed = probe.pack_weights(*wl0.slot_weights())
+        n_pools = min(64, max(2, math.ceil((1 << 30) / packed.numel())))
+        pools = [packed] + [packed.clone() for _ in range(n_pools - 1)]
+        del probe
+        for N in Ns:
+            T = G * N
+            buf = B.RankBuffers(T, 1, G, G, 1, d, f)
+            buf.topk_ids.copy_((torch.arange(T, device="cuda", dtype=torch.int32) % G).view(T, 1))
+            buf.topk_w.fill_(1.0)
+            buf.replica_map.copy_(torch.arange(G, device="cuda", dtype=torch.int32).view(G, 1))
+            buf.quota.fill_(N)
+            buf.x.copy_(torch.randn(T, d, generator=gen, device="cuda").to(torch.bfloat16))
+            graphs = _capture_graphs(torch, buf, pools)
+            s = buf.shape
+            ffn_graphs = []
+            for blob in pools:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
+                                        buf.status)
+                ffn_graphs.append(g)
+
+            def med(gs):
+                ts = []
+                for i in range(3):
+                    gs[i % n_pools].replay()
+                for i in range(replays):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    gs[i % n_pools].replay()
+                    b.record()
+                    b.synchronize()
+                    ts.append(a.elapsed_time(b) * 1e3)
+                return float(np.median(ts)), float(np.percentile(ts, 10)), float(np.percentile(ts, 90))
+
+            t_block, b10, b90 = med(graphs)
+            t_ffn, f10, f90 = med(ffn_graphs)
+            tiles = G * (-(-N // 128))
+            rows.append(dict(G=G, n=N, N=G * N, tiles=tiles, t_block_us=t_block, t_ffn_us=t_ffn, block_p10=b10,
+                             block_p90=b90, ffn_p10=f10, ffn_p90=f90, status=int(buf.status.item())))
+            print(json.dumps(rows[-1]), file=sys.stderr, flush=True)
+            del buf, graphs, ffn_graphs
+            torch.cuda.empty_cache()
+        del pools, packed
+        torch.cuda.empty_cache()
+    G = np.array([r["G"] for r in rows])
+    N = np.array([r["N"] for r in rows])
+    tiles = np.array([r["tiles"] for r in rows])
+    result = {"sweep": {"d": d, "f": f, "points": len(rows), "replays": replays}, "rows": rows}
+    for scope in ("ffn", "block"):
+        t = np.array([r[f"t_{scope}_us"] for r in rows])
+        result[f"fit_{scope}"] = C.fit_max_affine(G, N, t)
+        result[f"fit_{scope}_tile"] = C.fit_max_affine(G, N, t, tiles=tiles, tile_aware=True)
+    print(json.dumps(result))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--sweep-G", default="")
+    ap.add_argument("--sweep-N", default="")
+    ap.add_argument("--replays", type=int, default=30)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,211 @@
+// Host side of the C ABI: argument checks, tensor-map encoding, kernel launches.
+// Nothing here synchronises, allocates or reads device memory.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "tempo_kernels.cuh"
+
+namespace tempo {
+
+// ---- helpers ------------------------------------------------------------------------------------
+constexpr int kMaxE = 1024, kMaxG = 1024, kMaxR = 8, kMaxTopK = 32;
+
+static int check_shape(const tempo_shape* s) {
+  if (s == nullptr) return TEMPO_ERR_NULL;
+  if (s->T <= 0 || s->k <= 0 || s->E <= 0 || s->G_max <= 0 || s->R_max <= 0 || s->d <= 0 || s->f <= 0 || s->M_cap <= 0)
+    return TEMPO_ERR_SHAPE;
+  if (s->d % 128 || s->f % 128 || s->M_cap % 128) return TEMPO_ERR_SHAPE;
+  if (s->E > kMaxE || s->G_max > kMaxG || s->R_max > kMaxR || s->k > kMaxTopK) return TEMPO_ERR_UNSUPPORTED;
+  if (static_cast<long long>(s->T) * s->k > 0x7fff0000ll || static_cast<long long>(s->M_cap) > 0x7fff0000ll)
+    return TEMPO_ERR_UNSUPPORTED;
+  if (dispatch_smem_bytes(s->E, s->R_max, s->G_max) > 220 * 1024) return TEMPO_ERR_UNSUPPORTED;
+  return TEMPO_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;   // resolved once; a pure host-side driver routine
+  if (fn == nullptr) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// u8 matrix [rows, cols] row-major, box = 128 columns x box_rows rows, 128-byte swizzle.
+static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols};
+  const cuuint32_t box[2] = {128, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return n;
+}
+
+static int launch_gemm(int mode, const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
+                       const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y,
+                       uint32_t* status, cudaStream_t stream) {
+  const PackLayout L = pack_layout(s->G_max, s->d, s->f);
+  const uint8_t* blob = static_cast<const uint8_t*>(packed);
+  const int sms = sm_count();
+  if (sms <= 0) return TEMPO_ERR_CUDA;
+  CUtensorMap tmA, tmB;
+  GemmParams p{};
+  p.G_max = s->G_max;
+  p.M_cap = s->M_cap;
+  p.inst_off = inst_off;
+  p.m_pad = m_pad;
+  p.status = status;
+  p.sfa = a_sf;
+  if (mode == 0) {
+    const int K = s->d;
+    if (!make_map(&tmA, a_q, s->M_cap, K, 128)) return TEMPO_ERR_CUDA;
+    if (!make_map(&tmB, blob + L.off_w13, static_cast<uint64_t>(s->G_max) * 2 * s->f, K, 256)) return TEMPO_ERR_CUDA;
+    p.Kb = K / 128; p.JK = L.J1; p.NT = L.NT1; p.rowsB = 2 * s->f; p.n_cols = 2 * s->f;
+    p.ld_out = s->f; p.J_out = L.J2;
+    p.sfb = blob + L.off_sf13;
+    p.out_q = static_cast<uint8_t*>(h_q);
+    p.out_sf = h_sf;
+    return launch_ffn_gemm<0>(tmA, tmB, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+  }
+  const int K = s->f;
+  if (!make_map(&tmA, a_q, s->M_cap, K, 128)) return TEMPO_ERR_CUDA;
+  if (!make_map(&tmB, blob + L.off_w2, static_cast<uint64_t>(s->G_max) * s->d, K, 256)) return TEMPO_ERR_CUDA;
+  p.Kb = K / 128; p.JK = L.J2; p.NT = L.NT2; p.rowsB = s->d; p.n_cols = s->d;
+  p.ld_out = s->d; p.J_out = 0;
+  p.sfb = blob + L.off_sf2;
+  p.out_y = static_cast<__nv_bfloat16*>(y);
+  return launch_ffn_gemm<1>(tmA, tmB, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+}  // namespace tempo
+
+using namespace tempo;
+
+extern "C" {
+
+int tempo_version(void) { return 1; }
+
+const char* tempo_status_string(int code) {
+  switch (code) {
+    case TEMPO_OK: return "ok";
+    case TEMPO_ERR_NULL: return "a required pointer is NULL";
+    case TEMPO_ERR_SHAPE: return "a size is not positive or not a multiple of 128";
+    case TEMPO_ERR_UNSUPPORTED: return "a size exceeds a documented limit";
+    case TEMPO_ERR_CUDA: return "a CUDA call failed";
+    default: return "unknown code";
+  }
+}
+
+int tempo_m_cap_bound(const tempo_shape* s, int32_t* m_cap) {
+  if (s == nullptr || m_cap == nullptr) return TEMPO_ERR_NULL;
+  if (s->T <= 0 || s->k <= 0 || s->G_max <= 0) return TEMPO_ERR_SHAPE;
+  const long long v = ((static_cast<long long>(s->T) * s->k + 127) / 128) * 128 + 128ll * s->G_max;
+  if (v > 0x7fff0000ll) return TEMPO_ERR_UNSUPPORTED;
+  *m_cap = static_cast<int32_t>(v);
+  return TEMPO_OK;
+}
+
+int tempo_sf_bytes(int32_t rows, int32_t cols, size_t* bytes) {
+  if (bytes == nullptr) return TEMPO_ERR_NULL;
+  if (rows <= 0 || cols <= 0 || rows % 128 || cols % 128) return TEMPO_ERR_SHAPE;
+  *bytes = static_cast<size_t>(rows / 128) * (((cols / 128) + 3) / 4) * 512;
+  return TEMPO_OK;
+}
+
+int tempo_packed_weight_bytes(const tempo_shape* s, size_t* bytes) {
+  if (bytes == nullptr) return TEMPO_ERR_NULL;
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  *bytes = pack_layout(s->G_max, s->d, s->f).total;
+  return TEMPO_OK;
+}
+
+int tempo_pack_weights(const tempo_shape* s, const void* w13_q, const float* w13_s, const void* w2_q,
+                       const float* w2_s, void* packed, uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!w13_q || !w13_s || !w2_q || !w2_s || !packed || !status) return TEMPO_ERR_NULL;
+  return launch_pack(s->G_max, s->d, s->f, static_cast<const uint8_t*>(w13_q), w13_s,
+                     static_cast<const uint8_t*>(w2_q), w2_s, static_cast<uint8_t*>(packed), status,
+                     static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+int tempo_count_dispatch(const tempo_shape* s, const int32_t* topk_ids, const int32_t* n_valid,
+                         const int32_t* replica_map, const int32_t* quota, uint32_t* cum_counts,
+                         int32_t* counts, int32_t* inst_count, int32_t* inst_off, int32_t* pair_row,
+                         int32_t* row_pair, int32_t* tile_inst, int32_t* m_pad, uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!topk_ids || !replica_map || !quota || !counts || !inst_count || !inst_off || !pair_row || !row_pair ||
+      !tile_inst || !m_pad || !status)
+    return TEMPO_ERR_NULL;
+  DispatchParams p{s->T, s->k, s->E, s->G_max, s->R_max, s->M_cap, topk_ids, n_valid, replica_map, quota,
+                   cum_counts, counts, inst_count, inst_off, pair_row, row_pair, tile_inst, m_pad, status};
+  return launch_count_dispatch(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+int tempo_permute_pad(const tempo_shape* s, const void* x_bf16, const int32_t* row_pair, const int32_t* m_pad,
+                      void* a_q, uint8_t* a_sf, uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!x_bf16 || !row_pair || !m_pad || !a_q || !a_sf || !status) return TEMPO_ERR_NULL;
+  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, m_pad,
+                  static_cast<uint8_t*>(a_q), a_sf};
+  return launch_permute_pad(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+int tempo_ffn_gate_up(const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
+                      const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, uint32_t* status,
+                      void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!a_q || !a_sf || !packed || !inst_off || !m_pad || !h_q || !h_sf || !status) return TEMPO_ERR_NULL;
+  return launch_gemm(0, s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, nullptr, status,
+                     static_cast<cudaStream_t>(stream));
+}
+
+int tempo_ffn_down(const tempo_shape* s, const void* h_q, const uint8_t* h_sf, const void* packed,
+                   const int32_t* inst_off, const int32_t* m_pad, void* y_bf16, uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!h_q || !h_sf || !packed || !inst_off || !m_pad || !y_bf16 || !status) return TEMPO_ERR_NULL;
+  return launch_gemm(1, s, h_q, h_sf, packed, inst_off, m_pad, nullptr, nullptr, y_bf16, status,
+                     static_cast<cudaStream_t>(stream));
+}
+
+int tempo_grouped_ffn(const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
+                      const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y_bf16,
+                      uint32_t* status, void* stream) {
+  const int rc = tempo_ffn_gate_up(s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, status, stream);
+  if (rc != TEMPO_OK) return rc;
+  return tempo_ffn_down(s, h_q, h_sf, packed, inst_off, m_pad, y_bf16, status, stream);
+}
+
+int tempo_unpermute_combine(const tempo_shape* s, const void* y_bf16, const int32_t* pair_row, const float* topk_w,
+                            const int32_t* n_valid, void* out_bf16, uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!y_bf16 || !pair_row || !topk_w || !out_bf16 || !status) return TEMPO_ERR_NULL;
+  CombineParams p{s->T, s->k, s->d, static_cast<const __nv_bfloat16*>(y_bf16), pair_row, topk_w, n_valid,
+                  static_cast<__nv_bfloat16*>(out_bf16)};
+  return launch_combine(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+}  // extern "C"

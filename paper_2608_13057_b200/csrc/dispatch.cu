@@ -1,0 +1,210 @@
+// Step 1: fused count + quota dispatch + padded grouped layout, one CTA, one launch.
+//
+// The paper's in-graph contract (Section 4.4): dispatch through the replica table fused with
+// count collection into a cumulative per-expert counter, CUDA-graph padding rows masked, rows
+// renormalised at use, zero-sum row -> uniform over the replicas holding the expert.  Here the
+// table holds integer shares x_{e,r} (Eq. 2) that are honoured exactly and deterministically:
+// pairs of one expert are ranked by ascending pair index and cut into contiguous rank runs.
+//
+// Ranks come from scans, not from atomics, so the result is bit-reproducible:
+//   pass 1  every warp owns a contiguous range of pairs and builds its own histogram
+//           (__match_any_sync groups equal experts inside a 32-pair step);
+//   scan    per expert, an exclusive prefix over the 32 warp histograms gives each warp's base
+//           rank and the total n_e; the replica boundaries B_r follow from the quota row;
+//   pass 2  every warp walks its range again, rank = base + position among equal lanes.
+#include "tempo_kernels.cuh"
+
+namespace tempo {
+
+constexpr int kDispThreads = 1024;
+constexpr int kDispWarps = kDispThreads / 32;
+
+
+__global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const DispatchParams p) {
+  extern __shared__ int32_t smem[];
+  const int E = p.E, R = p.R_max, G = p.G_max;
+  int32_t* hist = smem;                       // [kDispWarps][E]  warp histograms -> exclusive bases
+  int32_t* bnd = hist + kDispWarps * E;       // [E][R]           cumulative rank boundaries B_r
+  int32_t* owner = bnd + E * R;               // [G]              first (e,r) entry naming the slot
+  int32_t* m_inst = owner + G;                // [G]              rows of each instance
+  int32_t* off = m_inst + G;                  // [G+1]            padded offsets (not clamped)
+  __shared__ uint32_t s_status;
+  __shared__ int32_t s_carry;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int nv = p.T;
+  if (p.n_valid != nullptr) nv = max(0, min(*p.n_valid, p.T));
+  const int P = nv * p.k;                     // live pairs
+  const int total_pairs = p.T * p.k;
+
+  for (int i = tid; i < kDispWarps * E; i += kDispThreads) hist[i] = 0;
+  for (int i = tid; i < G; i += kDispThreads) { owner[i] = 0x7fffffff; m_inst[i] = 0; }
+  if (tid == 0) s_status = 0;
+  __syncthreads();
+
+  // contiguous range of this warp, a multiple of 32 pairs long
+  const int per_warp = ((P + kDispWarps - 1) / kDispWarps + 31) & ~31;
+  const int w_begin = min(P, warp * per_warp), w_end = min(P, w_begin + per_warp);
+  uint32_t my_status = 0;
+
+  // ---- pass 1: warp histograms -------------------------------------------------------------
+  for (int base = w_begin; base < w_end; base += 32) {
+    const int pidx = base + lane;
+    int e = -1;
+    if (pidx < w_end) {
+      e = p.topk_ids[pidx];
+      if (e < 0 || e >= E) { my_status |= TEMPO_STATUS_BAD_ID; e = -1; }
+    }
+    const uint32_t same = __match_any_sync(0xffffffffu, e);
+    if (e >= 0 && lane == __ffs(same) - 1) hist[warp * E + e] += __popc(same);
+    __syncwarp();
+  }
+  // ---- which (e, r) owns each slot: the first entry in row-major order ----------------------
+  for (int idx = tid; idx < E * R; idx += kDispThreads) {
+    const int slot = p.replica_map[idx];
+    if (slot >= 0 && slot < G) atomicMin(&owner[slot], idx);
+    else if (slot != -1) my_status |= TEMPO_STATUS_BAD_TABLE;
+  }
+  __syncthreads();
+
+  // ---- per expert: totals, warp bases, replica boundaries -----------------------------------
+  for (int e = tid; e < E; e += kDispThreads) {
+    int run = 0;
+    for (int w = 0; w < kDispWarps; ++w) {
+      const int c = hist[w * E + e];
+      hist[w * E + e] = run;
+      run += c;
+    }
+    const int n_e = run;
+    p.counts[e] = n_e;
+    if (p.cum_counts != nullptr) atomicAdd(&p.cum_counts[e], static_cast<uint32_t>(n_e));
+
+    unsigned long long S = 0;
+    uint32_t vmask = 0;
+    for (int r = 0; r < R; ++r) {
+      const int idx = e * R + r;
+      const int slot = p.replica_map[idx];
+      const int x = p.quota[idx];
+      if (slot == -1) { if (x != 0) my_status |= TEMPO_STATUS_BAD_TABLE; continue; }
+      if (slot < 0 || slot >= G) continue;                       // flagged above
+      if (owner[slot] != idx) { my_status |= TEMPO_STATUS_BAD_TABLE; continue; }
+      vmask |= 1u << r;
+      if (x < 0) my_status |= TEMPO_STATUS_BAD_TABLE; else S += static_cast<unsigned long long>(x);
+    }
+    const bool uniform = (S == 0);
+    if (uniform) S = __popc(vmask);
+    unsigned long long C = 0;
+    int prev = 0;
+    for (int r = 0; r < R; ++r) {
+      const int idx = e * R + r;
+      const bool valid = (vmask >> r) & 1u;
+      if (valid) C += uniform ? 1ull : static_cast<unsigned long long>(max(p.quota[idx], 0));
+      const int B = S > 0 ? static_cast<int>(C * static_cast<unsigned long long>(n_e) / S) : 0;
+      bnd[idx] = B;
+      if (valid) m_inst[p.replica_map[idx]] = B - prev;
+      prev = B;
+    }
+  }
+  __syncthreads();
+
+  // ---- padded offsets: exclusive scan of 128*ceil(m/128) in ascending slot id (warp 0) -------
+  if (warp == 0) {
+    if (lane == 0) s_carry = 0;
+    __syncwarp();
+    for (int base = 0; base < G; base += 32) {
+      const int i = base + lane;
+      const int padded = i < G ? ((m_inst[i] + kTileM - 1) / kTileM) * kTileM : 0;
+      int incl = padded;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      const int carry = s_carry;
+      if (i < G) off[i] = carry + incl - padded;
+      __syncwarp();
+      if (lane == 31) s_carry = carry + incl;
+      __syncwarp();
+    }
+    if (lane == 0) off[G] = s_carry;
+  }
+  __syncthreads();
+
+  const int M_pad_full = off[G];
+  const int m_pad = min(M_pad_full, p.M_cap);
+  if (tid == 0) {
+    *p.m_pad = m_pad;
+    if (M_pad_full > p.M_cap) my_status |= TEMPO_STATUS_CAPACITY;
+  }
+  for (int i = tid; i <= G; i += kDispThreads) {
+    p.inst_off[i] = min(off[i], p.M_cap);
+    if (i < G) p.inst_count[i] = max(0, min(m_inst[i], p.M_cap - off[i]));
+  }
+  for (int row = tid; row < p.M_cap; row += kDispThreads) p.row_pair[row] = -1;
+  for (int q = P + tid; q < total_pairs; q += kDispThreads) p.pair_row[q] = -1;
+  for (int tau = tid; tau < p.M_cap / kTileM; tau += kDispThreads) {
+    const int row = tau * kTileM;
+    int inst = -1;
+    if (row < m_pad) {
+      int lo = 0, hi = G;                                        // first i with off[i+1] > row
+      while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (off[mid + 1] > row) hi = mid; else lo = mid + 1;
+      }
+      inst = lo;
+    }
+    p.tile_inst[tau] = inst;
+  }
+  __syncthreads();   // row_pair is pre-filled before any thread scatters into it
+
+  // ---- pass 2: stable ranks -> replica -> row -------------------------------------------------
+  for (int base = w_begin; base < w_end; base += 32) {
+    const int pidx = base + lane;
+    int e = -1;
+    if (pidx < w_end) {
+      e = p.topk_ids[pidx];
+      if (e < 0 || e >= E) e = -1;
+    }
+    const uint32_t same = __match_any_sync(0xffffffffu, e);
+    int j = 0;
+    if (e >= 0) j = hist[warp * E + e] + __popc(same & ((1u << lane) - 1u));
+    __syncwarp();
+    if (e >= 0 && lane == __ffs(same) - 1) hist[warp * E + e] += __popc(same);
+    __syncwarp();
+    if (pidx < w_end) {
+      int row = -1;
+      if (e >= 0) {
+        int prev = 0;
+        for (int r = 0; r < R; ++r) {
+          const int B = bnd[e * R + r];
+          if (j < B) {                                           // B only grows on valid columns
+            const int cand = off[p.replica_map[e * R + r]] + (j - prev);
+            if (cand < p.M_cap) row = cand;
+            break;
+          }
+          prev = B;
+        }
+      }
+      p.pair_row[pidx] = row;
+      if (row >= 0) p.row_pair[row] = pidx;
+    }
+  }
+
+  if (my_status) atomicOr(&s_status, my_status);
+  __syncthreads();
+  if (tid == 0 && s_status) atomicOr(p.status, s_status);
+}
+
+size_t dispatch_smem_bytes(int E, int R, int G) {
+  return sizeof(int32_t) * (static_cast<size_t>(kDispWarps) * E + static_cast<size_t>(E) * R + 3 * static_cast<size_t>(G) + 1);
+}
+
+cudaError_t launch_count_dispatch(const DispatchParams& p, cudaStream_t stream) {
+  const size_t smem = dispatch_smem_bytes(p.E, p.R_max, p.G_max);
+  cudaError_t e = cudaFuncSetAttribute(count_dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  count_dispatch_kernel<<<1, kDispThreads, smem, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace tempo

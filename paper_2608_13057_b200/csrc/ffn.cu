@@ -1,0 +1,359 @@
+// Step 3: fp8 grouped SwiGLU FFN on the 5th-generation tensor cores (sm_100a).
+//
+// Two launches of one persistent, warp-specialised kernel template:
+//   MODE 0  GU = A * W13p^T per 128x256 tile (128 gate + 128 up columns of one 128-column block
+//           of H), epilogue H = silu(gate) * up, re-quantised to e4m3 with a 1x128 power-of-two
+//           scale, written with its scale byte;
+//   MODE 1  Y = Hq * W2^T per 128x256 tile, epilogue converts to bf16.
+// This is the load-dependent term of the paper's cost model (Section 2.1, Eq. 1): with few rows
+// per instance the kernel streams every activated instance's weights once (the floor b per
+// instance), with many rows it is bound by the tensor pipe (beta per row, in 128-row tiles, Eq. 3).
+//
+// Per CTA (one per SM, 192 threads):
+//   warp 0     TMA producer: 128x128 A tile + 256x128 B tile per K-block into a 4-stage ring of
+//              128-byte-swizzled shared memory; every 4th K-block also brings one 512-byte scale
+//              atom of A and two of B (cp.async.bulk)
+//   warp 1     MMA issuer: tcgen05.cp moves scale atoms into tensor memory, then four
+//              tcgen05.mma.kind::mxf8f6f4.block_scale (M128 N256 K32) per K-block accumulate in
+//              tensor memory; tcgen05.commit releases the stage / publishes the accumulator
+//   warps 2-5  epilogue: tcgen05.ld the accumulator (one row per thread), math, global stores
+// Scales are UE8M0 per 128 K-elements; the MMA takes one scale byte per row (A) and per column
+// (B) for each K=32 step, so the four steps of a K-block select the same byte (scale id kb % 4).
+//
+// Every mbarrier wait is bounded: after kWaitLimitNs the CTA raises an abort flag, all roles
+// leave their loops, TEMPO_STATUS_TIMEOUT is set and tensor memory is freed.
+#include <cuda.h>
+
+#include "tempo_kernels.cuh"
+
+namespace tempo {
+
+constexpr int kStages = 4;
+constexpr int kBlockK = 128;
+constexpr int kBlockN = 256;
+constexpr int kABytes = kTileM * kBlockK;                 // 16 KB
+constexpr int kBBytes = kBlockN * kBlockK;                // 32 KB
+constexpr int kSfaBytes = 512;
+constexpr int kSfbBytes = 1024;
+constexpr int kStageBytes = kABytes + kBBytes + 2048;     // 51200, a multiple of 1024
+constexpr int kGemmThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr int kSfCol0 = 256;                              // scale slot s: A at 256+16s, B at 260+16s
+constexpr int kMaxSlots = 1024;
+constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 1024;
+
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  unsigned long long t0 = 0;
+  for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_cp_sf(uint32_t tmem_addr, uint64_t desc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(tmem_addr), "l"(desc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_mxf8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows of 128 bytes, groups of
+// 8 rows 1024 bytes apart (stride byte offset), descriptor version 1.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  return static_cast<uint64_t>((addr >> 4) & 0x3fffu) | (1ull << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// Descriptor of a 32-row x 16-byte scale atom (no swizzle, 8-row groups 128 bytes apart).
+__device__ __forceinline__ uint64_t smem_desc_sf(uint32_t addr) {
+  return static_cast<uint64_t>((addr >> 4) & 0x3fffu) | (static_cast<uint64_t>(128 >> 4) << 32) | (1ull << 46);
+}
+// Instruction descriptor of kind::mxf8f6f4.block_scale: A, B e4m3 (format 0), both K-major,
+// N >> 3 at bit 17, UE8M0 scales (bit 23), M >> 4 at bit 24; scale ids at bits 4 (B) and 29 (A).
+__device__ __forceinline__ uint32_t instr_desc(int sf_id) {
+  return (static_cast<uint32_t>(kBlockN >> 3) << 17) | (1u << 23) | (static_cast<uint32_t>(kTileM >> 4) << 24) |
+         (static_cast<uint32_t>(sf_id) << 29) | (static_cast<uint32_t>(sf_id) << 4);
+}
+
+struct WorkItem {
+  int inst, nt, row0;
+};
+
+// Items are ordered instance-major, then N-tile, then M-tile, so CTAs running at the same time
+// share B tiles through L2 and an instance's A rows stay L2-resident across its N-tiles.
+__device__ __forceinline__ WorkItem decode_item(int x, const int* toff, int G, int NT) {
+  int lo = 0, hi = G - 1;
+  while (lo < hi) {                       // first i with NT * toff[i+1] > x
+    const int mid = (lo + hi) >> 1;
+    if (NT * toff[mid + 1] > x) hi = mid; else lo = mid + 1;
+  }
+  const int local = x - NT * toff[lo];
+  const int Mi = toff[lo + 1] - toff[lo];
+  WorkItem w;
+  w.inst = lo;
+  w.nt = local / Mi;
+  w.row0 = (toff[lo] + local % Mi) * kTileM;
+  return w;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t s_full[kStages];
+  __shared__ __align__(8) uint64_t s_empty[kStages];
+  __shared__ __align__(8) uint64_t s_acc_full;
+  __shared__ __align__(8) uint64_t s_acc_empty;
+  __shared__ uint32_t s_tmem_base;
+  __shared__ int s_abort_storage;
+  __shared__ int s_toff[kMaxSlots + 1];
+  volatile int* s_abort = &s_abort_storage;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const int G = p.G_max;
+  const int m_pad = max(0, min(*p.m_pad, p.M_cap)) & ~(kTileM - 1);
+  const int total = (m_pad / kTileM) * p.NT;
+
+  for (int i = tid; i <= G; i += kGemmThreads) s_toff[i] = max(0, min(p.inst_off[i], m_pad)) >> 7;
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 1); mbar_init(smem_u32(&s_empty[s]), 1); }
+    mbar_init(smem_u32(&s_acc_full), 1);
+    mbar_init(smem_u32(&s_acc_empty), 4);
+    s_abort_storage = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                 "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = s_tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer ---------------------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int x = blockIdx.x; x < total && ok; x += gridDim.x) {
+        const WorkItem w = decode_item(x, s_toff, G, p.NT);
+        const uint8_t* sfa_src = p.sfa + static_cast<size_t>(w.row0 >> 7) * p.JK * kSfaBytes;
+        const uint8_t* sfb_src = p.sfb + (static_cast<size_t>(w.inst) * p.NT + w.nt) * p.JK * kSfbBytes;
+        const int b_row = w.inst * p.rowsB + w.nt * kBlockN;
+        for (int kb = 0; kb < p.Kb; ++kb) {
+          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
+          const uint32_t full = smem_u32(&s_full[stage]);
+          const uint32_t sA = smem_base + stage * kStageBytes, sB = sA + kABytes, sSF = sB + kBBytes;
+          const bool with_sf = (kb & 3) == 0;
+          mbar_arrive_expect_tx(full, kABytes + kBBytes + (with_sf ? kSfaBytes + kSfbBytes : 0));
+          tma_load_2d(sA, &tmA, full, kb * kBlockK, w.row0);
+          tma_load_2d(sB, &tmB, full, kb * kBlockK, b_row);
+          if (with_sf) {
+            bulk_load(sSF, sfa_src + static_cast<size_t>(kb >> 2) * kSfaBytes, kSfaBytes, full);
+            bulk_load(sSF + kSfaBytes, sfb_src + static_cast<size_t>(kb >> 2) * kSfbBytes, kSfbBytes, full);
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer -----------------------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int x = blockIdx.x; x < total && ok; x += gridDim.x) {
+        if (!mbar_wait(smem_u32(&s_acc_empty), acc_phase ^ 1u, s_abort)) break;
+        tc_fence_after();
+        for (int kb = 0; kb < p.Kb; ++kb) {
+          if (!mbar_wait(smem_u32(&s_full[stage]), phase, s_abort)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sA = smem_base + stage * kStageBytes, sB = sA + kABytes, sSF = sB + kBBytes;
+          const uint32_t sfa_t = tmem_base + kSfCol0 + 16u * ((kb >> 2) & 1);
+          const uint32_t sfb_t = sfa_t + 4;
+          if ((kb & 3) == 0) {
+            tc_cp_sf(sfa_t, smem_desc_sf(sSF));
+            tc_cp_sf(sfb_t, smem_desc_sf(sSF + kSfaBytes));
+            tc_cp_sf(sfb_t + 4, smem_desc_sf(sSF + kSfaBytes + 512));
+          }
+          const uint32_t idesc = instr_desc(kb & 3);
+          const uint64_t da = smem_desc_sw128(sA), db = smem_desc_sw128(sB);
+#pragma unroll
+          for (int ks = 0; ks < kBlockK / 32; ++ks)
+            tc_mma_mxf8(tmem_base, da + 2u * ks, db + 2u * ks, idesc, sfa_t, sfb_t, (kb | ks) != 0 ? 1u : 0u);
+          tc_commit(smem_u32(&s_empty[stage]));
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit(smem_u32(&s_acc_full));
+        acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ------------------------------- epilogue --------------------------------------------------
+    const int quad = warp & 3;                       // tensor-memory lanes this warp may read
+    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+    uint32_t acc_phase = 0;
+    for (int x = blockIdx.x; x < total; x += gridDim.x) {
+      const WorkItem w = decode_item(x, s_toff, G, p.NT);
+      const int row = w.row0 + quad * 32 + lane;
+      if (!mbar_wait(smem_u32(&s_acc_full), acc_phase, s_abort)) break;
+      acc_phase ^= 1u;
+      tc_fence_after();
+      if constexpr (MODE == 0) {
+        float h[128];
+        float amax = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t g[32], u[32];
+          tmem_ld32(taddr + c * 32, g);
+          tmem_ld32(taddr + 128 + c * 32, u);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float gv = __uint_as_float(g[i]), uv = __uint_as_float(u[i]);
+            const float hv = __fdividef(gv, 1.f + __expf(-gv)) * uv;
+            h[c * 32 + i] = hv;
+            amax = fmaxf(amax, fabsf(hv));
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));
+        const int eps = pow2_scale_exponent(amax);
+        const float inv = pow2_neg(eps);
+        uint8_t* dst = p.out_q + static_cast<size_t>(row) * p.ld_out + w.nt * 128;
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+          uint4 q;
+          q.x = cvt_e4m3x4(h[16 * v + 0] * inv, h[16 * v + 1] * inv, h[16 * v + 2] * inv, h[16 * v + 3] * inv);
+          q.y = cvt_e4m3x4(h[16 * v + 4] * inv, h[16 * v + 5] * inv, h[16 * v + 6] * inv, h[16 * v + 7] * inv);
+          q.z = cvt_e4m3x4(h[16 * v + 8] * inv, h[16 * v + 9] * inv, h[16 * v + 10] * inv, h[16 * v + 11] * inv);
+          q.w = cvt_e4m3x4(h[16 * v + 12] * inv, h[16 * v + 13] * inv, h[16 * v + 14] * inv, h[16 * v + 15] * inv);
+          *reinterpret_cast<uint4*>(dst + 16 * v) = q;
+        }
+        p.out_sf[sf_index(row, w.nt, p.J_out)] = static_cast<uint8_t>(eps + 127);
+      } else {
+        __nv_bfloat16* dst = p.out_y + static_cast<size_t>(row) * p.ld_out + w.nt * kBlockN;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (w.nt * kBlockN + c * 32 < p.n_cols) {         // warp-uniform
+            uint32_t a[32];
+            tmem_ld32(taddr + c * 32, a);
+            tmem_wait_ld();
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              uint4 o;
+              uint32_t* ou = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(a[8 * v + 2 * i]),
+                                                               __uint_as_float(a[8 * v + 2 * i + 1]));
+                ou[i] = *reinterpret_cast<const uint32_t*>(&b);
+              }
+              *reinterpret_cast<uint4*>(dst + c * 32 + 8 * v) = o;
+            }
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (*s_abort) {
+    if (tid == 0) atomicOr(p.status, static_cast<uint32_t>(TEMPO_STATUS_TIMEOUT));
+    for (int i = 0; i < 50; ++i) __nanosleep(1000);  // let copies and MMAs in flight drain
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    __syncwarp();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+template <int MODE>
+cudaError_t launch_ffn_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, int num_sms,
+                            cudaStream_t stream) {
+  cudaError_t e = cudaFuncSetAttribute(ffn_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(kGemmSmemBytes));
+  if (e != cudaSuccess) return e;
+  const int max_items = (p.M_cap / kTileM) * p.NT;
+  const int grid = max(1, min(num_sms, max_items));
+  ffn_gemm_kernel<MODE><<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(tmA, tmB, p);
+  return cudaGetLastError();
+}
+
+template cudaError_t launch_ffn_gemm<0>(const CUtensorMap&, const CUtensorMap&, const GemmParams&, int, cudaStream_t);
+template cudaError_t launch_ffn_gemm<1>(const CUtensorMap&, const CUtensorMap&, const GemmParams&, int, cudaStream_t);
+
+}  // namespace tempo

@@ -1,0 +1,72 @@
+// Parameter blocks and launchers shared between the kernel files and the C-ABI host code.
+#pragma once
+
+#include <cuda.h>
+
+#include "tempo_common.cuh"
+
+namespace tempo {
+
+struct DispatchParams {
+  int T, k, E, G_max, R_max, M_cap;
+  const int32_t* topk_ids;
+  const int32_t* n_valid;
+  const int32_t* replica_map;
+  const int32_t* quota;
+  uint32_t* cum_counts;
+  int32_t* counts;
+  int32_t* inst_count;
+  int32_t* inst_off;
+  int32_t* pair_row;
+  int32_t* row_pair;
+  int32_t* tile_inst;
+  int32_t* m_pad;
+  uint32_t* status;
+};
+size_t dispatch_smem_bytes(int E, int R, int G);
+cudaError_t launch_count_dispatch(const DispatchParams& p, cudaStream_t stream);
+
+struct PermuteParams {
+  int k, d, M_cap;
+  const __nv_bfloat16* x;
+  const int32_t* row_pair;
+  const int32_t* m_pad;
+  uint8_t* a_q;
+  uint8_t* a_sf;
+};
+cudaError_t launch_permute_pad(const PermuteParams& p, cudaStream_t stream);
+
+struct CombineParams {
+  int T, k, d;
+  const __nv_bfloat16* y;
+  const int32_t* pair_row;
+  const float* topk_w;
+  const int32_t* n_valid;
+  __nv_bfloat16* out;
+};
+cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream);
+
+struct PackLayout {
+  size_t off_w13, off_w2, off_sf13, off_sf2, total;
+  int J1, J2, NT1, NT2;
+};
+PackLayout pack_layout(int G, int d, int f);
+cudaError_t launch_pack(int G, int d, int f, const uint8_t* w13_q, const float* w13_s, const uint8_t* w2_q,
+                        const float* w2_s, uint8_t* packed, uint32_t* status, cudaStream_t stream);
+
+struct GemmParams {
+  int Kb, JK, NT, rowsB, n_cols, G_max, M_cap, ld_out, J_out;
+  const uint8_t* sfa;
+  const uint8_t* sfb;
+  const int32_t* inst_off;
+  const int32_t* m_pad;
+  uint8_t* out_q;
+  uint8_t* out_sf;
+  __nv_bfloat16* out_y;
+  uint32_t* status;
+};
+template <int MODE>
+cudaError_t launch_ffn_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, int num_sms,
+                            cudaStream_t stream);
+
+}  // namespace tempo

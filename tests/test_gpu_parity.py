@@ -1,0 +1,289 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs.
+
+Bars: integer / index / byte outputs of count+dispatch and permute+quantise are bit-exact (fp8 codes
+modulo the sign of zero); FFN outputs are within max|err| <= 2e-2 * max|ref| and
+mean|err| / mean|ref| <= 5e-3 of the oracle evaluated on the same dequantised fp8 values.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import tempo_oracle as O
+from paper_2608_13057_b200 import workloads as W
+from tests.gpu_util import codes_equal_mod_signed_zero, dispatch_outputs, sf_decode, to_np
+
+pytestmark = pytest.mark.gpu
+
+MAX_TOL, MEAN_TOL = 2e-2, 5e-3
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2608_13057_b200 import binding
+    return binding
+
+
+def _dispatch_only(B, wl, M_cap=None, cum=None):
+    """Run step 1 alone with small feature dims (the step does not touch them)."""
+    buf = B.RankBuffers(wl.T, wl.k, wl.E, wl.G_max, wl.R_max, 128, 128, M_cap=M_cap)
+    buf.topk_ids.copy_(torch.from_numpy(wl.topk_ids))
+    buf.n_valid.fill_(int(wl.n_valid))
+    buf.replica_map.copy_(torch.from_numpy(wl.replica_map))
+    buf.quota.copy_(torch.from_numpy(wl.quota))
+    if cum is not None:
+        buf.cum_counts.copy_(torch.from_numpy(cum.view(np.int32)))
+    B.tempo_count_dispatch(buf.shape, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts,
+                           buf.counts, buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair, buf.tile_inst,
+                           buf.m_pad, buf.status)
+    torch.cuda.synchronize()
+    return buf, dispatch_outputs(buf)
+
+
+def _assert_dispatch_equal(got, ref):
+    for key in ("counts", "inst_count", "inst_off", "pair_row", "row_pair", "tile_inst"):
+        assert np.array_equal(got[key], ref[key]), key
+    assert got["m_pad"] == int(ref["m_pad"])
+    assert got["status"] == int(ref["status"])
+    if "cum_counts" in ref:
+        assert np.array_equal(got["cum_counts"], ref["cum_counts"])
+
+
+def _table_case(ids, n_valid, rmap, quota, G_max, name="table"):
+    ids = np.asarray(ids, np.int32)
+    T, k = ids.shape
+    rmap = np.asarray(rmap, np.int32)
+    E, R = rmap.shape
+    return W.Workload(name, T, k, E, G_max, R, 128, 128, n_valid, ids, np.ones((T, k), np.float32), rmap,
+                      np.asarray(quota, np.int32), np.full(G_max, -1, np.int32), None, 0, 0)
+
+
+def _dispatch_cases():
+    yield W.config1()
+    yield W.config2()
+    yield W.config2(n_valid=200)
+    for c in ("uniform", "token_balanced", "hot_whole"):
+        yield W.config3(c)
+    yield W.config4(with_x=False)
+    yield W.config5_point(4, 129, with_x=False)
+    yield W.config5_point(64, 4096, with_x=False)           # 262144 pairs, the largest sweep point
+    yield W.config5_point(1, 1, with_x=False)
+    for s in range(8):
+        yield W.random_small(200 + s)
+    for s in range(4):
+        yield W.random_small(300 + s, T=200, E=37, k=3, stale=True)   # stale rows: sum != n_e
+    yield W.random_small(17, T=9, n_valid=5)
+    yield W.random_small(18, T=9, n_valid=0)
+    yield W.random_small(19, T=9, n_valid=1)
+    g = np.random.default_rng(9)
+    # all pairs to one expert, three replicas, zero-sum row -> uniform fallback
+    yield _table_case(np.zeros((301, 1)), 301, [[0, 1, 2]], [[0, 0, 0]], 3, "zero-sum")
+    # share on a -1 column, slot out of range, negative share, slot claimed twice, ids out of range
+    yield _table_case(np.zeros((50, 1)), 50, [[0, -1, 2]], [[10, 25, 15]], 4, "share-on-missing")
+    yield _table_case(np.zeros((40, 1)), 40, [[0, 9, 1]], [[20, 10, 20]], 4, "slot-out-of-range")
+    yield _table_case(np.zeros((40, 1)), 40, [[0, 1, -1]], [[-5, 40, 0]], 4, "negative-share")
+    yield _table_case([[0], [1], [1], [0]], 4, [[0], [0]], [[2], [2]], 1, "slot-claimed-twice")
+    yield _table_case([[0], [5], [-1], [0]], 4, [[0]], [[2]], 1, "bad-ids")
+    # an expert with n_e = 0 but a non-zero share; duplicate expert inside one token; E not a multiple of 32
+    ids = g.integers(1, 37, size=(64, 4))
+    ids[:, 1] = ids[:, 0]
+    rmap = np.full((37, 2), -1)
+    rmap[:20, 0] = np.arange(20)
+    rmap[:5, 1] = 20 + np.arange(5)
+    quota = g.integers(0, 30, size=(37, 2))
+    yield _table_case(ids, 64, rmap, quota * (rmap >= 0), 25, "dup-in-token")
+    for m in (127, 128, 129):
+        yield _table_case(np.zeros((m, 1)), m, [[0]], [[m]], 1, f"tile-{m}")
+
+
+@pytest.mark.parametrize("wl", list(_dispatch_cases()), ids=lambda w: w.name)
+def test_count_dispatch_bit_exact(B, wl):
+    cum = np.full(wl.E, 2 ** 32 - 5, np.uint32)
+    buf, got = _dispatch_only(B, wl, cum=cum)
+    ref = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, buf.M_cap, cum_counts=cum)
+    _assert_dispatch_equal(got, ref)
+
+
+def test_count_dispatch_capacity_overflow(B):
+    ids = (np.arange(600, dtype=np.int32) % 2).reshape(600, 1)
+    wl = _table_case(ids, 600, [[0], [1]], [[300], [300]], 2, "capacity")
+    buf, got = _dispatch_only(B, wl, M_cap=640)
+    ref = O.count_dispatch(wl.topk_ids, 600, wl.replica_map, wl.quota, 2, 640)
+    _assert_dispatch_equal(got, ref)
+    assert got["status"] & B.STATUS_CAPACITY
+
+
+def test_count_dispatch_is_deterministic_and_accumulates(B):
+    wl = W.config3("token_balanced")
+    buf, first = _dispatch_only(B, wl)
+    for _ in range(20):
+        B.tempo_count_dispatch(buf.shape, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts,
+                               buf.counts, buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair, buf.tile_inst,
+                               buf.m_pad, buf.status)
+    torch.cuda.synchronize()
+    again = dispatch_outputs(buf)
+    for key in ("counts", "pair_row", "row_pair", "inst_off"):
+        assert np.array_equal(first[key], again[key])
+    assert np.array_equal(again["cum_counts"], (21 * first["counts"].astype(np.uint64) % 2 ** 32).astype(np.uint32))
+
+
+# ---------------------------------------------------------------------------------------------------
+
+def _run_block(B, wl, M_cap=None):
+    buf = B.RankBuffers.for_workload(wl, M_cap=M_cap)
+    buf.run_block()
+    torch.cuda.synchronize()
+    return buf
+
+
+def _check_permute(buf, ref):
+    m_pad = int(ref["m_pad"])
+    a_q = to_np(buf.a_q)[:m_pad]
+    a_s = sf_decode(to_np(buf.a_sf), buf.M_cap, buf.d)[:m_pad]
+    assert codes_equal_mod_signed_zero(a_q, ref["a_q"][:m_pad]).all()
+    assert np.array_equal(a_s, ref["a_s"][:m_pad])
+
+
+def _err(got, ref):
+    got = np.asarray(got, np.float64)
+    ref = np.asarray(ref, np.float64)
+    scale = np.abs(ref).max()
+    return np.abs(got - ref).max() / max(scale, 1e-30), np.abs(got - ref).mean() / max(np.abs(ref).mean(), 1e-30)
+
+
+def _small_block_cases():
+    yield W.config1()
+    yield W.config5_point(1, 40, d=256, f=256)
+    yield W.config5_point(3, 129, d=384, f=640)           # two tiles per instance, odd block counts
+    for s in range(3):
+        yield W.random_small(400 + s, T=40, E=6, k=2, d=256, f=384)
+    yield W.random_small(410, T=40, n_valid=23)
+
+
+@pytest.mark.parametrize("wl", list(_small_block_cases()), ids=lambda w: w.name)
+def test_block_matches_oracle_elementwise(B, wl):
+    buf = _run_block(B, wl)
+    ref = O.expert_block(wl, M_cap=buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    _check_permute(buf, ref)
+    m_pad = int(ref["m_pad"])
+    # H: compare dequantised values (a code may differ where fp32 accumulation crosses a rounding boundary)
+    h_gpu = O.dequantise_1x128(to_np(buf.h_q)[:m_pad], sf_decode(to_np(buf.h_sf), buf.M_cap, buf.f)[:m_pad])
+    h_ref = O.dequantise_1x128(ref["h_q"][:m_pad], ref["h_s"][:m_pad])
+    if m_pad:
+        mx, mean = _err(h_gpu, h_ref)
+        assert mx <= 0.07 and mean <= MEAN_TOL, ("H", mx, mean)
+        mx, mean = _err(to_np(buf.y)[:m_pad], ref["y"][:m_pad])
+        assert mx <= MAX_TOL and mean <= MEAN_TOL, ("Y", mx, mean)
+    out = to_np(buf.out)
+    mx, mean = _err(out[:wl.n_valid], ref["out"][:wl.n_valid])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("out", mx, mean)
+    assert np.all(out[wl.n_valid:] == 0)
+    assert np.all(out[(ref["pair_row"].reshape(wl.T, wl.k) < 0).all(1)] == 0)
+    assert not (int(buf.status.item()) & B.STATUS_TIMEOUT)
+
+
+def test_flat_decode_config_full(B):
+    wl = W.config2()
+    buf = _run_block(B, wl)
+    ref = O.expert_block(wl, M_cap=buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    _check_permute(buf, ref)
+    m_pad = int(ref["m_pad"])
+    mx, mean = _err(to_np(buf.y)[:m_pad], ref["y"][:m_pad])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("Y", mx, mean)
+    mx, mean = _err(to_np(buf.out), ref["out"])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("out", mx, mean)
+    # masking variant: rows >= n_valid are CUDA-graph padding
+    wl2 = W.config2(n_valid=200)
+    buf2 = _run_block(B, wl2)
+    ref2 = O.expert_block(wl2, M_cap=buf2.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf2), ref2)
+    mx, mean = _err(to_np(buf2.out)[:200], ref2["out"][:200])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL
+    assert torch.all(buf2.out[200:] == 0)
+
+
+def _sampled_rows_check(B, wl, buf, rows_per_inst=6, n_tokens=48, seed=0):
+    """Full-size check on sampled outputs the oracle computes one by one."""
+    ref = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    g = np.random.default_rng(seed)
+    tokens = np.sort(g.choice(wl.n_valid, size=min(n_tokens, wl.n_valid), replace=False))
+    need = set()
+    pr = ref["pair_row"].reshape(wl.T, wl.k)
+    for t in tokens:
+        need.update(int(r) for r in pr[t] if r >= 0)
+    for i in range(wl.G_max):
+        lo, m = int(ref["inst_off"][i]), int(ref["inst_count"][i])
+        if m == 0:
+            continue
+        picks = {lo, lo + m - 1, lo + min(m - 1, 127), lo + min(m - 1, 128)}
+        picks.update(int(v) for v in lo + g.integers(0, m, size=rows_per_inst))
+        need.update(picks)
+    rows = np.array(sorted(need))
+    inst_of = np.searchsorted(ref["inst_off"][1:], rows, side="right")
+    y_ref = np.zeros((len(rows), wl.d), np.float32)
+    a_q_gpu = to_np(buf.a_q[torch.from_numpy(rows).cuda()])
+    a_s_gpu = sf_decode(to_np(buf.a_sf), buf.M_cap, buf.d)[rows]
+    for i in np.unique(inst_of):
+        sel = np.nonzero(inst_of == i)[0]
+        toks = ref["row_pair"][rows[sel]] // wl.k
+        a_q, a_s = O.quantise_1x128(wl.x[toks])
+        assert codes_equal_mod_signed_zero(a_q_gpu[sel], a_q).all() and np.array_equal(a_s_gpu[sel], a_s)
+        w = wl.expert_weights(int(wl.slot_expert[i]))
+        _, _, y_ref[sel] = O.expert_ffn(a_q, a_s, w.w13_q, w.w13_s, w.w2_q, w.w2_s)
+    y_gpu = to_np(buf.y[torch.from_numpy(rows).cuda()])
+    mx, mean = _err(y_gpu, y_ref)
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("Y rows", mx, mean)
+    # combine on the sampled tokens, from the oracle's own Y rows
+    pos = {int(r): n for n, r in enumerate(rows)}
+    out_ref = np.zeros((len(tokens), wl.d), np.float32)
+    for n, t in enumerate(tokens):
+        acc = np.zeros(wl.d, np.float32)
+        for s in range(wl.k):
+            if pr[t, s] >= 0:
+                acc = acc + wl.topk_w[t, s] * y_ref[pos[int(pr[t, s])]]
+        out_ref[n] = acc
+    out_gpu = to_np(buf.out[torch.from_numpy(tokens).cuda()])
+    mx, mean = _err(out_gpu, out_ref)
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("out rows", mx, mean)
+    assert not (int(buf.status.item()) & B.STATUS_TIMEOUT)
+
+
+def test_mixed_config_three_splits_sampled_and_split_invariant(B):
+    outs = []
+    for case in ("uniform", "token_balanced", "hot_whole"):
+        wl = W.config3(case)
+        buf = _run_block(B, wl)
+        _sampled_rows_check(B, wl, buf)
+        outs.append(buf.out.clone())
+        del buf
+    # replicas hold copies of the same weights and a row's result does not depend on where it sits
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+
+
+def test_prefill_config_sampled(B):
+    wl = W.config4()
+    buf = _run_block(B, wl)
+    _sampled_rows_check(B, wl, buf, rows_per_inst=3, n_tokens=16)
+
+
+@pytest.mark.parametrize("G,N", [(1, 1), (2, 129), (8, 512), (64, 64)])
+def test_sweep_points_sampled(B, G, N):
+    wl = W.config5_point(G, N)
+    buf = _run_block(B, wl)
+    _sampled_rows_check(B, wl, buf, rows_per_inst=2, n_tokens=8)
+
+
+def test_pack_rejects_non_power_of_two_scales(B):
+    wl = W.config1()
+    buf = B.RankBuffers(wl.T, wl.k, wl.E, wl.G_max, wl.R_max, wl.d, wl.f)
+    w13_q, w13_s, w2_q, w2_s = wl.slot_weights()
+    buf.pack_weights(w13_q, w13_s, w2_q, w2_s)
+    assert int(buf.status.item()) == 0
+    w2_s = w2_s.copy()
+    w2_s[0, 0, 0] = 0.3
+    buf.pack_weights(w13_q, w13_s, w2_q, w2_s)
+    assert int(buf.status.item()) & B.STATUS_BAD_SCALE
