@@ -391,7 +391,7 @@ def run_sweep(args):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
                     B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
-                                        buf.status)
+                                        buf.status, buf.workspace)
                 ffn_graphs.append(g)
 
             def med(gs):

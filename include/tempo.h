@@ -80,6 +80,14 @@ int tempo_m_cap_bound(const tempo_shape* shape /*[host]*/, int32_t* m_cap /*[hos
 /* [host] Bytes of a scale-byte buffer for an operand of `rows` x `cols` (see sf_index above). */
 int tempo_sf_bytes(int32_t rows, int32_t cols, size_t* bytes /*[host]*/);
 
+/*
+ * [host] Bytes of the scratch buffer of tempo_grouped_ffn: two int32 counters per 128-row tile of
+ * the padded layout (8 * M_cap / 128, rounded up to 256).  The caller allocates it and ZEROES it
+ * once; every call that completes leaves it zero again.  After a call that reported
+ * TEMPO_STATUS_TIMEOUT zero it again.  Calls that may overlap on the GPU need a buffer each.
+ */
+int tempo_workspace_bytes(const tempo_shape* shape /*[host]*/, size_t* bytes /*[host]*/);
+
 /* [host] Bytes of the packed weight blob for G_max instances of shape (d, f). */
 int tempo_packed_weight_bytes(const tempo_shape* shape /*[host]*/, size_t* bytes /*[host]*/);
 
@@ -137,7 +145,11 @@ int tempo_permute_pad(const tempo_shape* shape, const void* x_bf16, const int32_
  * by the MMA), H = silu(gate) * up, then H is re-quantised like step 2 along f.
  *   in   a_q, a_sf, packed, inst_off, m_pad    out  h_q u8 [M_cap, f], h_sf u8 [tempo_sf_bytes(M_cap, f)]
  * Step 3b: Y = Hq * W2^T, stored as bf16.       out  y bf16 [M_cap, d]
- * tempo_grouped_ffn runs 3a then 3b.  Rows >= m_pad are not written.
+ * tempo_grouped_ffn runs 3a and 3b in ONE kernel: the down tiles of a 128-row tile start as soon as
+ * its H blocks are complete (tracked in `workspace`, see tempo_workspace_bytes), so the weight
+ * stream never pauses between the two GEMMs.  The kernel's CTAs wait for each other's H blocks
+ * (bounded, one per SM): launch it on a GPU it does not have to share with another long-running
+ * kernel, or the wait may time out (TEMPO_STATUS_TIMEOUT).  Rows >= m_pad are not written.
  */
 int tempo_ffn_gate_up(const tempo_shape* shape, const void* a_q, const uint8_t* a_sf, const void* packed,
                       const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf,
@@ -146,7 +158,7 @@ int tempo_ffn_down(const tempo_shape* shape, const void* h_q, const uint8_t* h_s
                    const int32_t* inst_off, const int32_t* m_pad, void* y_bf16, uint32_t* status, void* stream);
 int tempo_grouped_ffn(const tempo_shape* shape, const void* a_q, const uint8_t* a_sf, const void* packed,
                       const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y_bf16,
-                      uint32_t* status, void* stream);
+                      uint32_t* status, void* workspace, void* stream);
 
 /*
  * Step 4.  out[t,:] = sum_{s<k, pair_row[t*k+s] >= 0} topk_w[t,s] * y[pair_row[t*k+s], :], slots in

@@ -12,13 +12,14 @@ from typing import Optional
 
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtempo.so")
+_LIB_PATH = os.environ.get("TEMPO_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libtempo.so")
 
 TEMPO_OK = 0
 STATUS_BAD_ID, STATUS_BAD_TABLE, STATUS_CAPACITY, STATUS_TIMEOUT, STATUS_BAD_SCALE = 1, 2, 4, 8, 16
 
 EXPORTS = (
-    "tempo_version", "tempo_status_string", "tempo_m_cap_bound", "tempo_sf_bytes", "tempo_packed_weight_bytes",
+    "tempo_version", "tempo_status_string", "tempo_m_cap_bound", "tempo_sf_bytes", "tempo_workspace_bytes",
+    "tempo_packed_weight_bytes",
     "tempo_pack_weights", "tempo_count_dispatch", "tempo_permute_pad", "tempo_ffn_gate_up", "tempo_ffn_down",
     "tempo_grouped_ffn", "tempo_unpermute_combine",
 )
@@ -90,6 +91,12 @@ def tempo_sf_bytes(rows: int, cols: int) -> int:
     return out.value
 
 
+def tempo_workspace_bytes(shape: TempoShape) -> int:
+    out = ctypes.c_size_t(0)
+    _check(_lib.tempo_workspace_bytes(ctypes.byref(shape), ctypes.byref(out)), "tempo_workspace_bytes")
+    return out.value
+
+
 def tempo_packed_weight_bytes(shape: TempoShape) -> int:
     out = ctypes.c_size_t(0)
     _check(_lib.tempo_packed_weight_bytes(ctypes.byref(shape), ctypes.byref(out)), "tempo_packed_weight_bytes")
@@ -131,11 +138,12 @@ def tempo_ffn_down(shape, h_q, h_sf, packed, inst_off, m_pad, y_bf16, status):
                                _ptr(y_bf16, torch.bfloat16), _ptr(status, torch.int32), _stream()), "tempo_ffn_down")
 
 
-def tempo_grouped_ffn(shape, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status):
+def tempo_grouped_ffn(shape, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, workspace):
     _check(_lib.tempo_grouped_ffn(ctypes.byref(shape), _ptr(a_q, torch.uint8), _ptr(a_sf, torch.uint8),
                                   _ptr(packed, torch.uint8), _ptr(inst_off, torch.int32), _ptr(m_pad, torch.int32),
                                   _ptr(h_q, torch.uint8), _ptr(h_sf, torch.uint8), _ptr(y_bf16, torch.bfloat16),
-                                  _ptr(status, torch.int32), _stream()), "tempo_grouped_ffn")
+                                  _ptr(status, torch.int32), _ptr(workspace, torch.uint8), _stream()),
+           "tempo_grouped_ffn")
 
 
 def tempo_unpermute_combine(shape, y_bf16, pair_row, topk_w, n_valid, out_bf16, status):
@@ -181,6 +189,7 @@ class RankBuffers:
         self.h_sf = torch.full((tempo_sf_bytes(self.M_cap, f),), 127, **u8)
         self.y = torch.zeros(self.M_cap, d, dtype=torch.bfloat16, device=dev)
         self.out = torch.zeros(T, d, dtype=torch.bfloat16, device=dev)
+        self.workspace = torch.zeros(tempo_workspace_bytes(self.shape), **u8)   # counters start at zero
         self.packed = None
 
     def pack_weights(self, w13_q, w13_s, w2_q, w2_s):
@@ -201,7 +210,7 @@ class RankBuffers:
                              self.tile_inst, self.m_pad, self.status)
         tempo_permute_pad(s, self.x, self.row_pair, self.m_pad, self.a_q, self.a_sf, self.status)
         tempo_grouped_ffn(s, self.a_q, self.a_sf, packed, self.inst_off, self.m_pad, self.h_q, self.h_sf, self.y,
-                          self.status)
+                          self.status, self.workspace)
         tempo_unpermute_combine(s, self.y, self.pair_row, self.topk_w, self.n_valid, self.out, self.status)
 
     def upload(self, wl, with_weights=True):

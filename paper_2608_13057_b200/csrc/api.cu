@@ -58,40 +58,36 @@ static int sm_count() {
   return n;
 }
 
-static int launch_gemm(int mode, const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
-                       const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y,
-                       uint32_t* status, cudaStream_t stream) {
+// run_mask bit 0: gate/up tiles, bit 1: down tiles.  Buffers a side does not use may be NULL.
+static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
+                           const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y,
+                           uint32_t* status, void* workspace, cudaStream_t stream) {
   const PackLayout L = pack_layout(s->G_max, s->d, s->f);
   const uint8_t* blob = static_cast<const uint8_t*>(packed);
   const int sms = sm_count();
   if (sms <= 0) return TEMPO_ERR_CUDA;
-  CUtensorMap tmA, tmB;
-  GemmParams p{};
+  CUtensorMap tmA1, tmA2;
+  // a side that does not run still needs a well-formed map; point it at a buffer that exists
+  if (!make_map(&tmA1, (run_mask & 1) ? a_q : h_q, s->M_cap, (run_mask & 1) ? s->d : s->f, 128)) return TEMPO_ERR_CUDA;
+  if (!make_map(&tmA2, h_q, s->M_cap, s->f, 128)) return TEMPO_ERR_CUDA;
+  FfnParams p{};
+  p.side[0] = GemmSide{s->d / 128, L.J1, L.NT1, blob + L.off_w13, a_sf, blob + L.off_sf13};
+  p.side[1] = GemmSide{s->f / 128, L.J2, L.NT2, blob + L.off_w2, h_sf, blob + L.off_sf2};
+  p.run_mask = run_mask;
   p.G_max = s->G_max;
   p.M_cap = s->M_cap;
+  p.d = s->d;
+  p.f = s->f;
+  p.J_h = L.J2;
   p.inst_off = inst_off;
   p.m_pad = m_pad;
+  p.h_q = static_cast<uint8_t*>(h_q);
+  p.h_sf = h_sf;
+  p.y = static_cast<__nv_bfloat16*>(y);
+  p.ready = static_cast<int32_t*>(workspace);
+  p.done = p.ready ? p.ready + s->M_cap / 128 : nullptr;
   p.status = status;
-  p.sfa = a_sf;
-  if (mode == 0) {
-    const int K = s->d;
-    if (!make_map(&tmA, a_q, s->M_cap, K, 128)) return TEMPO_ERR_CUDA;
-    if (!make_map(&tmB, blob + L.off_w13, static_cast<uint64_t>(s->G_max) * 2 * s->f, K, 256)) return TEMPO_ERR_CUDA;
-    p.Kb = K / 128; p.JK = L.J1; p.NT = L.NT1; p.rowsB = 2 * s->f; p.n_cols = 2 * s->f;
-    p.ld_out = s->f; p.J_out = L.J2;
-    p.sfb = blob + L.off_sf13;
-    p.out_q = static_cast<uint8_t*>(h_q);
-    p.out_sf = h_sf;
-    return launch_ffn_gemm<0>(tmA, tmB, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
-  }
-  const int K = s->f;
-  if (!make_map(&tmA, a_q, s->M_cap, K, 128)) return TEMPO_ERR_CUDA;
-  if (!make_map(&tmB, blob + L.off_w2, static_cast<uint64_t>(s->G_max) * s->d, K, 256)) return TEMPO_ERR_CUDA;
-  p.Kb = K / 128; p.JK = L.J2; p.NT = L.NT2; p.rowsB = s->d; p.n_cols = s->d;
-  p.ld_out = s->d; p.J_out = 0;
-  p.sfb = blob + L.off_sf2;
-  p.out_y = static_cast<__nv_bfloat16*>(y);
-  return launch_ffn_gemm<1>(tmA, tmB, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+  return launch_ffn(tmA1, tmA2, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
 
 }  // namespace tempo
@@ -126,6 +122,14 @@ int tempo_sf_bytes(int32_t rows, int32_t cols, size_t* bytes) {
   if (bytes == nullptr) return TEMPO_ERR_NULL;
   if (rows <= 0 || cols <= 0 || rows % 128 || cols % 128) return TEMPO_ERR_SHAPE;
   *bytes = static_cast<size_t>(rows / 128) * (((cols / 128) + 3) / 4) * 512;
+  return TEMPO_OK;
+}
+
+int tempo_workspace_bytes(const tempo_shape* s, size_t* bytes) {
+  if (bytes == nullptr) return TEMPO_ERR_NULL;
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  *bytes = ffn_workspace_bytes(s->M_cap);
   return TEMPO_OK;
 }
 
@@ -177,8 +181,8 @@ int tempo_ffn_gate_up(const tempo_shape* s, const void* a_q, const uint8_t* a_sf
   const int rc = check_shape(s);
   if (rc != TEMPO_OK) return rc;
   if (!a_q || !a_sf || !packed || !inst_off || !m_pad || !h_q || !h_sf || !status) return TEMPO_ERR_NULL;
-  return launch_gemm(0, s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, nullptr, status,
-                     static_cast<cudaStream_t>(stream));
+  return launch_ffn_host(1, s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, nullptr, status, nullptr,
+                         static_cast<cudaStream_t>(stream));
 }
 
 int tempo_ffn_down(const tempo_shape* s, const void* h_q, const uint8_t* h_sf, const void* packed,
@@ -186,16 +190,19 @@ int tempo_ffn_down(const tempo_shape* s, const void* h_q, const uint8_t* h_sf, c
   const int rc = check_shape(s);
   if (rc != TEMPO_OK) return rc;
   if (!h_q || !h_sf || !packed || !inst_off || !m_pad || !y_bf16 || !status) return TEMPO_ERR_NULL;
-  return launch_gemm(1, s, h_q, h_sf, packed, inst_off, m_pad, nullptr, nullptr, y_bf16, status,
-                     static_cast<cudaStream_t>(stream));
+  return launch_ffn_host(2, s, nullptr, nullptr, packed, inst_off, m_pad, const_cast<void*>(h_q),
+                         const_cast<uint8_t*>(h_sf), y_bf16, status, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int tempo_grouped_ffn(const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
                       const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y_bf16,
-                      uint32_t* status, void* stream) {
-  const int rc = tempo_ffn_gate_up(s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, status, stream);
+                      uint32_t* status, void* workspace, void* stream) {
+  const int rc = check_shape(s);
   if (rc != TEMPO_OK) return rc;
-  return tempo_ffn_down(s, h_q, h_sf, packed, inst_off, m_pad, y_bf16, status, stream);
+  if (!a_q || !a_sf || !packed || !inst_off || !m_pad || !h_q || !h_sf || !y_bf16 || !status || !workspace)
+    return TEMPO_ERR_NULL;
+  return launch_ffn_host(3, s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, workspace,
+                         static_cast<cudaStream_t>(stream));
 }
 
 int tempo_unpermute_combine(const tempo_shape* s, const void* y_bf16, const int32_t* pair_row, const float* topk_w,

@@ -1,55 +1,63 @@
 // Step 4: weighted un-permute.  out[t,:] = sum over the token's k slots, in slot order, of
 // topk_w[t,s] * y[pair_row[t,s],:] with fp32 accumulation and a bf16 store (the "combine" of
-// Section 2.1 restricted to this rank's partial sum).  HBM-bound gather: one CTA per token,
+// Section 2.1 restricted to this rank's partial sum).  HBM-bound gather with
 // 16-byte loads and stores.
 #include "tempo_kernels.cuh"
 
 namespace tempo {
 
-constexpr int kCombThreads = 128;
-constexpr int kMaxK = 32;
+constexpr int kCombThreads = 256;
 
-
+// One thread per (token, 8 columns).  The k row indices and weights are read first, then all
+// gathers of a group of 8 slots are issued before any is consumed, so the thread pays the memory
+// latency once per group instead of once per slot; the sum itself stays in slot order.
 __global__ void __launch_bounds__(kCombThreads) combine_kernel(const CombineParams p) {
-  __shared__ int32_t s_row[kMaxK];
-  __shared__ float s_w[kMaxK];
   const int t = blockIdx.x;
+  const int col = (blockIdx.y * kCombThreads + threadIdx.x) * 8;
+  if (col >= p.d) return;
   int nv = p.T;
   if (p.n_valid != nullptr) nv = max(0, min(*p.n_valid, p.T));
-  if (threadIdx.x < p.k) {
-    const int idx = t * p.k + threadIdx.x;
-    s_row[threadIdx.x] = t < nv ? p.pair_row[idx] : -1;
-    s_w[threadIdx.x] = p.topk_w[idx];
-  }
-  __syncthreads();
-  __nv_bfloat16* dst = p.out + static_cast<size_t>(t) * p.d;
-  for (int col = threadIdx.x * 8; col < p.d; col += kCombThreads * 8) {
-    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    for (int s = 0; s < p.k; ++s) {
-      const int row = s_row[s];
-      if (row < 0) continue;
-      const float w = s_w[s];
-      const uint4 v = *reinterpret_cast<const uint4*>(p.y + static_cast<size_t>(row) * p.d + col);
-      const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  if (t < nv) {
+    for (int s0 = 0; s0 < p.k; s0 += 8) {
+      int row[8];
+      float w[8];
+      uint4 v[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        acc[2 * i] = fmaf(w, __uint_as_float(u[i] << 16), acc[2 * i]);
-        acc[2 * i + 1] = fmaf(w, __uint_as_float(u[i] & 0xffff0000u), acc[2 * i + 1]);
+      for (int i = 0; i < 8; ++i) {
+        const int s = s0 + i;
+        row[i] = s < p.k ? __ldg(p.pair_row + t * p.k + s) : -1;
+        w[i] = s < p.k ? __ldg(p.topk_w + t * p.k + s) : 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        v[i] = row[i] >= 0 ? __ldg(reinterpret_cast<const uint4*>(p.y + static_cast<size_t>(row[i]) * p.d + col))
+                           : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (row[i] < 0) continue;
+        const uint32_t u[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[2 * j] = fmaf(w[i], __uint_as_float(u[j] << 16), acc[2 * j]);
+          acc[2 * j + 1] = fmaf(w[i], __uint_as_float(u[j] & 0xffff0000u), acc[2 * j + 1]);
+        }
       }
     }
-    uint4 o;
-    uint32_t* ou = reinterpret_cast<uint32_t*>(&o);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const __nv_bfloat162 b = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
-      ou[i] = *reinterpret_cast<const uint32_t*>(&b);
-    }
-    *reinterpret_cast<uint4*>(dst + col) = o;
   }
+  uint4 o;
+  uint32_t* ou = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __nv_bfloat162 b = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+    ou[i] = *reinterpret_cast<const uint32_t*>(&b);
+  }
+  *reinterpret_cast<uint4*>(p.out + static_cast<size_t>(t) * p.d + col) = o;
 }
 
 cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream) {
-  combine_kernel<<<p.T, kCombThreads, 0, stream>>>(p);
+  const dim3 grid(p.T, (p.d / 8 + kCombThreads - 1) / kCombThreads);
+  combine_kernel<<<grid, kCombThreads, 0, stream>>>(p);
   return cudaGetLastError();
 }
 

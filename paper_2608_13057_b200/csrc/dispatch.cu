@@ -28,6 +28,8 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
   int32_t* owner = bnd + E * R;               // [G]              first (e,r) entry naming the slot
   int32_t* m_inst = owner + G;                // [G]              rows of each instance
   int32_t* off = m_inst + G;                  // [G+1]            padded offsets (not clamped)
+  int32_t* rmap_s = off + G + 1;              // [E][R]           replica_map, staged once
+  int32_t* quota_s = rmap_s + E * R;          // [E][R]           quota, staged once
   __shared__ uint32_t s_status;
   __shared__ int32_t s_carry;
 
@@ -37,6 +39,9 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
   const int P = nv * p.k;                     // live pairs
   const int total_pairs = p.T * p.k;
 
+  // all table reads are issued up front, together with the first ids, so the kernel pays the
+  // global-memory latency once
+  for (int i = tid; i < E * R; i += kDispThreads) { rmap_s[i] = p.replica_map[i]; quota_s[i] = p.quota[i]; }
   for (int i = tid; i < kDispWarps * E; i += kDispThreads) hist[i] = 0;
   for (int i = tid; i < G; i += kDispThreads) { owner[i] = 0x7fffffff; m_inst[i] = 0; }
   if (tid == 0) s_status = 0;
@@ -52,7 +57,7 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
     const int pidx = base + lane;
     int e = -1;
     if (pidx < w_end) {
-      e = p.topk_ids[pidx];
+      e = __ldg(p.topk_ids + pidx);
       if (e < 0 || e >= E) { my_status |= TEMPO_STATUS_BAD_ID; e = -1; }
     }
     const uint32_t same = __match_any_sync(0xffffffffu, e);
@@ -61,7 +66,7 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
   }
   // ---- which (e, r) owns each slot: the first entry in row-major order ----------------------
   for (int idx = tid; idx < E * R; idx += kDispThreads) {
-    const int slot = p.replica_map[idx];
+    const int slot = rmap_s[idx];
     if (slot >= 0 && slot < G) atomicMin(&owner[slot], idx);
     else if (slot != -1) my_status |= TEMPO_STATUS_BAD_TABLE;
   }
@@ -83,8 +88,8 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
     uint32_t vmask = 0;
     for (int r = 0; r < R; ++r) {
       const int idx = e * R + r;
-      const int slot = p.replica_map[idx];
-      const int x = p.quota[idx];
+      const int slot = rmap_s[idx];
+      const int x = quota_s[idx];
       if (slot == -1) { if (x != 0) my_status |= TEMPO_STATUS_BAD_TABLE; continue; }
       if (slot < 0 || slot >= G) continue;                       // flagged above
       if (owner[slot] != idx) { my_status |= TEMPO_STATUS_BAD_TABLE; continue; }
@@ -98,10 +103,10 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
     for (int r = 0; r < R; ++r) {
       const int idx = e * R + r;
       const bool valid = (vmask >> r) & 1u;
-      if (valid) C += uniform ? 1ull : static_cast<unsigned long long>(max(p.quota[idx], 0));
+      if (valid) C += uniform ? 1ull : static_cast<unsigned long long>(max(quota_s[idx], 0));
       const int B = S > 0 ? static_cast<int>(C * static_cast<unsigned long long>(n_e) / S) : 0;
       bnd[idx] = B;
-      if (valid) m_inst[p.replica_map[idx]] = B - prev;
+      if (valid) m_inst[rmap_s[idx]] = B - prev;
       prev = B;
     }
   }
@@ -161,7 +166,7 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
     const int pidx = base + lane;
     int e = -1;
     if (pidx < w_end) {
-      e = p.topk_ids[pidx];
+      e = __ldg(p.topk_ids + pidx);
       if (e < 0 || e >= E) e = -1;
     }
     const uint32_t same = __match_any_sync(0xffffffffu, e);
@@ -177,7 +182,7 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
         for (int r = 0; r < R; ++r) {
           const int B = bnd[e * R + r];
           if (j < B) {                                           // B only grows on valid columns
-            const int cand = off[p.replica_map[e * R + r]] + (j - prev);
+            const int cand = off[rmap_s[e * R + r]] + (j - prev);
             if (cand < p.M_cap) row = cand;
             break;
           }
@@ -195,7 +200,7 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
 }
 
 size_t dispatch_smem_bytes(int E, int R, int G) {
-  return sizeof(int32_t) * (static_cast<size_t>(kDispWarps) * E + static_cast<size_t>(E) * R + 3 * static_cast<size_t>(G) + 1);
+  return sizeof(int32_t) * (static_cast<size_t>(kDispWarps) * E + 3 * static_cast<size_t>(E) * R + 3 * static_cast<size_t>(G) + 1);
 }
 
 cudaError_t launch_count_dispatch(const DispatchParams& p, cudaStream_t stream) {

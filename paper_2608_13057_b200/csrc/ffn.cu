@@ -1,18 +1,25 @@
-// Step 3: fp8 grouped SwiGLU FFN on the 5th-generation tensor cores (sm_100a).
+// Step 3: fp8 grouped SwiGLU FFN on the 5th-generation tensor cores (sm_100a), ONE persistent kernel.
 //
-// Two launches of one persistent, warp-specialised kernel template:
-//   MODE 0  GU = A * W13p^T per 128x256 tile (128 gate + 128 up columns of one 128-column block
-//           of H), epilogue H = silu(gate) * up, re-quantised to e4m3 with a 1x128 power-of-two
-//           scale, written with its scale byte;
-//   MODE 1  Y = Hq * W2^T per 128x256 tile, epilogue converts to bf16.
+// Two kinds of 128x256 output tiles:
+//   gate/up  GU = A * W13t^T (128 gate + 128 up columns of one 128-column block of H), epilogue
+//            H = silu(gate) * up, re-quantised to e4m3 with a 1x128 power-of-two scale;
+//   down     Y = Hq * W2t^T, epilogue converts to bf16.
 // This is the load-dependent term of the paper's cost model (Section 2.1, Eq. 1): with few rows
 // per instance the kernel streams every activated instance's weights once (the floor b per
 // instance), with many rows it is bound by the tensor pipe (beta per row, in 128-row tiles, Eq. 3).
+// Both kinds run in the same launch so the weight stream has one ramp and one tail and the CTAs
+// that run out of gate/up tiles go straight on to down tiles.  A down tile needs every H block
+// of its 128 rows: the epilogue warps of a finished gate/up tile bump a per-M-tile counter, and
+// only the ACTIVATION loads of a down tile wait for it (bounded); its weight loads never wait,
+// so HBM keeps streaming.  The counters clean themselves: the last down tile of an M-tile to see
+// the counter complete puts it back to zero.
 //
-// Per CTA (one per SM, 192 threads):
-//   warp 0     TMA producer: 128x128 A tile + 256x128 B tile per K-block into a 4-stage ring of
-//              128-byte-swizzled shared memory; every 4th K-block also brings one 512-byte scale
-//              atom of A and two of B (cp.async.bulk)
+// Per CTA (one per SM, 256 threads):
+//   warp 0     weight producer: per K-block one contiguous 32 KB bulk copy of a pre-swizzled
+//              packed B tile (+ two 512-byte scale atoms every 4th K-block) into a 4-stage ring
+//   warp 6     activation producer: per K-block a 128x128 A tile (TMA tensor copy, 128-byte
+//              swizzle) (+ one scale atom every 4th K-block); waits for H where needed
+//   warp 7     dependency scout: runs ahead of warp 6 through the down tiles, watches the H counters
 //   warp 1     MMA issuer: tcgen05.cp moves scale atoms into tensor memory, then four
 //              tcgen05.mma.kind::mxf8f6f4.block_scale (M128 N256 K32) per K-block accumulate in
 //              tensor memory; tcgen05.commit releases the stage / publishes the accumulator
@@ -20,8 +27,8 @@
 // Scales are UE8M0 per 128 K-elements; the MMA takes one scale byte per row (A) and per column
 // (B) for each K=32 step, so the four steps of a K-block select the same byte (scale id kb % 4).
 //
-// Every mbarrier wait is bounded: after kWaitLimitNs the CTA raises an abort flag, all roles
-// leave their loops, TEMPO_STATUS_TIMEOUT is set and tensor memory is freed.
+// Every wait is bounded: after kWaitLimitNs the CTA raises an abort flag, all roles leave their
+// loops, TEMPO_STATUS_TIMEOUT is set and tensor memory is freed.
 #include <cuda.h>
 
 #include "tempo_kernels.cuh"
@@ -36,7 +43,8 @@ constexpr int kBBytes = kBlockN * kBlockK;                // 32 KB
 constexpr int kSfaBytes = 512;
 constexpr int kSfbBytes = 1024;
 constexpr int kStageBytes = kABytes + kBBytes + 2048;     // 51200, a multiple of 1024
-constexpr int kGemmThreads = 192;
+constexpr int kGemmThreads = 256;
+constexpr int kTileOverhead = 5;                          // per-tile fixed cost in K-block steps (ramp + epilogue)
 constexpr int kTmemCols = 512;
 constexpr int kSfCol0 = 256;                              // scale slot s: A at 256+16s, B at 260+16s
 constexpr int kMaxSlots = 1024;
@@ -91,6 +99,15 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
                : "memory");
 }
+// Same copy with an L2 evict-first hint: for weight tiles that are read once per launch.
+__device__ __forceinline__ void bulk_load_stream(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar), "l"(policy)
+      : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -140,12 +157,13 @@ __device__ __forceinline__ uint32_t instr_desc(int sf_id) {
 }
 
 struct WorkItem {
-  int inst, nt, row0;
+  int side;      // 0 gate/up, 1 down
+  int inst, nt, row0, m_tiles;   // m_tiles: M-tiles of the instance (how often its B tiles are re-read)
 };
 
-// Items are ordered instance-major, then N-tile, then M-tile, so CTAs running at the same time
-// share B tiles through L2 and an instance's A rows stay L2-resident across its N-tiles.
-__device__ __forceinline__ WorkItem decode_item(int x, const int* toff, int G, int NT) {
+// Tiles of one side are numbered instance-major, then N-tile, then M-tile, so CTAs running at the
+// same time share B tiles through L2 and an instance's A rows stay L2-resident across its N-tiles.
+__device__ __forceinline__ WorkItem decode_item(int side, int x, const int* toff, int G, int NT) {
   int lo = 0, hi = G - 1;
   while (lo < hi) {                       // first i with NT * toff[i+1] > x
     const int mid = (lo + hi) >> 1;
@@ -154,15 +172,56 @@ __device__ __forceinline__ WorkItem decode_item(int x, const int* toff, int G, i
   const int local = x - NT * toff[lo];
   const int Mi = toff[lo + 1] - toff[lo];
   WorkItem w;
+  w.side = side;
   w.inst = lo;
   w.nt = local / Mi;
   w.row0 = (toff[lo] + local % Mi) * kTileM;
+  w.m_tiles = Mi;
   return w;
 }
 
-template <int MODE>
+// Static tile assignment, the same arithmetic in every role of every CTA.
+//   gate/up tiles: x = c, c + C, ...  (n1 tiles; the first r1 = n1 % C CTAs get one more)
+//   down tiles:    dealt in rounds.  The CTAs WITHOUT the extra gate/up tile ("light") take part
+//                  in every round, the others only from round `lead` on, where `lead` is the extra
+//                  tile's cost in down tiles - so every CTA streams about the same bytes.
+struct TileIter {
+  int c, C, n1, n2, r1, light, lead;
+  int i1, round;
+  __device__ TileIter(int c_, int C_, int n1_, int n2_, int Kb1, int Kb2) {
+    c = c_; C = C_; n1 = n1_; n2 = n2_;
+    r1 = n1 % C;
+    light = C - r1;
+    lead = (r1 == 0 || n2 == 0) ? 0 : (2 * (Kb1 + kTileOverhead) + (Kb2 + kTileOverhead)) / (2 * (Kb2 + kTileOverhead));
+    i1 = c; round = 0;
+  }
+  // side and tile number of this CTA's next tile; false when it has none left
+  __device__ bool next(int& side, int& x) {
+    if (i1 < n1) { side = 0; x = i1; i1 += C; return true; }
+    for (;;) {
+      int y;
+      if (round < lead) {
+        if (c < r1) { round = lead; continue; }           // heavy CTAs skip the lead rounds
+        y = round * light + (c - r1);
+      } else {
+        y = lead * light + (round - lead) * C + c;
+      }
+      ++round;
+      if (y >= n2) return false;
+      side = 1; x = y;
+      return true;
+    }
+  }
+};
+
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
 __global__ void __launch_bounds__(kGemmThreads, 1)
-ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmParams p) {
+ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2, const FfnParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t s_full[kStages];
   __shared__ __align__(8) uint64_t s_empty[kStages];
@@ -170,21 +229,28 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   __shared__ __align__(8) uint64_t s_acc_empty;
   __shared__ uint32_t s_tmem_base;
   __shared__ int s_abort_storage;
+  __shared__ int s_dep_storage;
   __shared__ int s_toff[kMaxSlots + 1];
   volatile int* s_abort = &s_abort_storage;
+  volatile int* s_dep = &s_dep_storage;   // down tiles of this CTA whose H rows are known complete
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int G = p.G_max;
   const int m_pad = max(0, min(*p.m_pad, p.M_cap)) & ~(kTileM - 1);
-  const int total = (m_pad / kTileM) * p.NT;
+  const int m_tiles = m_pad / kTileM;
+  const int n1 = (p.run_mask & 1) ? m_tiles * p.side[0].NT : 0;
+  const int n2 = (p.run_mask & 2) ? m_tiles * p.side[1].NT : 0;
+  const bool fused = p.run_mask == 3;
+  const int Kb1 = p.side[0].Kb, Kb2 = p.side[1].Kb;
 
   for (int i = tid; i <= G; i += kGemmThreads) s_toff[i] = max(0, min(p.inst_off[i], m_pad)) >> 7;
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 1); mbar_init(smem_u32(&s_empty[s]), 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 2); mbar_init(smem_u32(&s_empty[s]), 1); }
     mbar_init(smem_u32(&s_acc_full), 1);
     mbar_init(smem_u32(&s_acc_empty), 4);
     s_abort_storage = 0;
+    s_dep_storage = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -199,29 +265,103 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const uint32_t tmem_base = s_tmem_base;
 
   if (warp == 0) {
-    // ------------------------------- TMA producer ---------------------------------------------
+    // ------------------------------- weight producer ------------------------------------------
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
       bool ok = true;
-      for (int x = blockIdx.x; x < total && ok; x += gridDim.x) {
-        const WorkItem w = decode_item(x, s_toff, G, p.NT);
-        const uint8_t* sfa_src = p.sfa + static_cast<size_t>(w.row0 >> 7) * p.JK * kSfaBytes;
-        const uint8_t* sfb_src = p.sfb + (static_cast<size_t>(w.inst) * p.NT + w.nt) * p.JK * kSfbBytes;
-        const int b_row = w.inst * p.rowsB + w.nt * kBlockN;
-        for (int kb = 0; kb < p.Kb; ++kb) {
+      TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+      int side, x;
+      while (ok && it.next(side, x)) {
+        const GemmSide& gs = p.side[side];
+        const WorkItem w = decode_item(side, x, s_toff, G, gs.NT);
+        const uint8_t* sfb_src = gs.sfb + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.JK * kSfbBytes;
+        const uint8_t* b_src = gs.wt + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.Kb * kBBytes;
+        const bool stream_b = w.m_tiles <= 2;
+        for (int kb = 0; kb < gs.Kb; ++kb) {
           if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
           const uint32_t full = smem_u32(&s_full[stage]);
-          const uint32_t sA = smem_base + stage * kStageBytes, sB = sA + kABytes, sSF = sB + kBBytes;
+          const uint32_t sB = smem_base + stage * kStageBytes + kABytes, sSF = sB + kBBytes;
           const bool with_sf = (kb & 3) == 0;
-          mbar_arrive_expect_tx(full, kABytes + kBBytes + (with_sf ? kSfaBytes + kSfbBytes : 0));
-          tma_load_2d(sA, &tmA, full, kb * kBlockK, w.row0);
-          tma_load_2d(sB, &tmB, full, kb * kBlockK, b_row);
-          if (with_sf) {
-            bulk_load(sSF, sfa_src + static_cast<size_t>(kb >> 2) * kSfaBytes, kSfaBytes, full);
-            bulk_load(sSF + kSfaBytes, sfb_src + static_cast<size_t>(kb >> 2) * kSfbBytes, kSfbBytes, full);
-          }
+          mbar_arrive_expect_tx(full, kBBytes + (with_sf ? kSfbBytes : 0));
+          if (stream_b) bulk_load_stream(sB, b_src + static_cast<size_t>(kb) * kBBytes, kBBytes, full);
+          else bulk_load(sB, b_src + static_cast<size_t>(kb) * kBBytes, kBBytes, full);
+          if (with_sf) bulk_load(sSF + kSfaBytes, sfb_src + static_cast<size_t>(kb >> 2) * kSfbBytes, kSfbBytes, full);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
+      }
+    }
+  } else if (warp == 6) {
+    // ------------------------------- activation producer --------------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      int n_down = 0;
+      bool ok = true;
+      TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+      int side, x;
+      while (ok && it.next(side, x)) {
+        const GemmSide& gs = p.side[side];
+        const WorkItem w = decode_item(side, x, s_toff, G, gs.NT);
+        const uint8_t* sfa_src = gs.sfa + static_cast<size_t>(w.row0 >> 7) * gs.JK * kSfaBytes;
+        const CUtensorMap* tm = side == 0 ? &tmA1 : &tmA2;
+        if (side == 1 && fused) {
+          // wait until the scout (warp 7) has seen every H block of these 128 rows complete
+          ++n_down;
+          unsigned long long t0 = 0;
+          for (uint32_t spin = 0; *s_dep < n_down; ++spin) {
+            if ((spin & 255u) == 255u) {
+              if (*s_abort) { ok = false; break; }
+              const unsigned long long now = global_timer_ns();
+              if (t0 == 0) t0 = now;
+              else if (now - t0 > kWaitLimitNs) { *s_abort = 1; ok = false; break; }
+            }
+          }
+          if (!ok) break;
+          __threadfence();
+          asm volatile("fence.proxy.async;" ::: "memory");   // H was written by ordinary stores, TMA reads it
+        }
+        for (int kb = 0; kb < gs.Kb; ++kb) {
+          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
+          const uint32_t full = smem_u32(&s_full[stage]);
+          const uint32_t sA = smem_base + stage * kStageBytes, sSF = sA + kABytes + kBBytes;
+          const bool with_sf = (kb & 3) == 0;
+          mbar_arrive_expect_tx(full, kABytes + (with_sf ? kSfaBytes : 0));
+          tma_load_2d(sA, tm, full, kb * kBlockK, w.row0);
+          if (with_sf) bulk_load(sSF, sfa_src + static_cast<size_t>(kb >> 2) * kSfaBytes, kSfaBytes, full);
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 7) {
+    // ------------------------------- dependency scout -----------------------------------------
+    // Runs ahead through this CTA's down tiles: waits (bounded) until the four epilogue warps of
+    // every gate/up tile of the tile's 128 rows have published their H rows, then tells the
+    // activation producer through s_dep.  The last down tile of an M-tile to get here puts the
+    // two global counters back to zero, so the workspace is clean when the kernel ends.
+    if (lane == 0 && fused) {
+      TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+      int side, x, cleared = 0;
+      const int want = 4 * p.side[0].NT;
+      bool ok = true;
+      while (ok && it.next(side, x)) {
+        if (side == 0) continue;
+        const WorkItem w = decode_item(1, x, s_toff, G, p.side[1].NT);
+        const int tau = w.row0 >> 7;
+        unsigned long long t0 = 0;
+        for (uint32_t spin = 0; ld_acquire(p.ready + tau) < want; ++spin) {
+          if ((spin & 63u) == 63u) {
+            if (*s_abort) { ok = false; break; }
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) { *s_abort = 1; ok = false; break; }
+          }
+        }
+        if (!ok) break;
+        if (atomicAdd(p.done + tau, 1) == p.side[1].NT - 1) {
+          atomicExch(p.ready + tau, 0);
+          atomicExch(p.done + tau, 0);
+        }
+        __threadfence();
+        *s_dep = ++cleared;
       }
     }
   } else if (warp == 1) {
@@ -229,10 +369,13 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (lane == 0) {
       uint32_t stage = 0, phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int x = blockIdx.x; x < total && ok; x += gridDim.x) {
+      TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+      int side, x;
+      while (ok && it.next(side, x)) {
+        const int Kb = p.side[side].Kb;
         if (!mbar_wait(smem_u32(&s_acc_empty), acc_phase ^ 1u, s_abort)) break;
         tc_fence_after();
-        for (int kb = 0; kb < p.Kb; ++kb) {
+        for (int kb = 0; kb < Kb; ++kb) {
           if (!mbar_wait(smem_u32(&s_full[stage]), phase, s_abort)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sA = smem_base + stage * kStageBytes, sB = sA + kABytes, sSF = sB + kBBytes;
@@ -255,18 +398,20 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         acc_phase ^= 1u;
       }
     }
-  } else {
+  } else if (warp >= 2 && warp <= 5) {
     // ------------------------------- epilogue --------------------------------------------------
     const int quad = warp & 3;                       // tensor-memory lanes this warp may read
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
     uint32_t acc_phase = 0;
-    for (int x = blockIdx.x; x < total; x += gridDim.x) {
-      const WorkItem w = decode_item(x, s_toff, G, p.NT);
+    TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+    int side, x;
+    while (it.next(side, x)) {
+      const WorkItem w = decode_item(side, x, s_toff, G, p.side[side].NT);
       const int row = w.row0 + quad * 32 + lane;
       if (!mbar_wait(smem_u32(&s_acc_full), acc_phase, s_abort)) break;
       acc_phase ^= 1u;
       tc_fence_after();
-      if constexpr (MODE == 0) {
+      if (side == 0) {
         float h[128];
         float amax = 0.f;
 #pragma unroll
@@ -285,10 +430,10 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));
+        if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));   // accumulator drained: the next tile may start
         const int eps = pow2_scale_exponent(amax);
         const float inv = pow2_neg(eps);
-        uint8_t* dst = p.out_q + static_cast<size_t>(row) * p.ld_out + w.nt * 128;
+        uint8_t* dst = p.h_q + static_cast<size_t>(row) * p.f + w.nt * 128;
 #pragma unroll
         for (int v = 0; v < 8; ++v) {
           uint4 q;
@@ -298,32 +443,39 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           q.w = cvt_e4m3x4(h[16 * v + 12] * inv, h[16 * v + 13] * inv, h[16 * v + 14] * inv, h[16 * v + 15] * inv);
           *reinterpret_cast<uint4*>(dst + 16 * v) = q;
         }
-        p.out_sf[sf_index(row, w.nt, p.J_out)] = static_cast<uint8_t>(eps + 127);
+        p.h_sf[sf_index(row, w.nt, p.J_h)] = static_cast<uint8_t>(eps + 127);
+        if (fused) {                                  // publish this warp's 32 rows of the H block
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) atomicAdd(p.ready + (w.row0 >> 7), 1);
+        }
       } else {
-        __nv_bfloat16* dst = p.out_y + static_cast<size_t>(row) * p.ld_out + w.nt * kBlockN;
+        // drain the accumulator into packed bf16 registers first, release it, then store
+        uint32_t packed[128];
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-          if (w.nt * kBlockN + c * 32 < p.n_cols) {         // warp-uniform
-            uint32_t a[32];
-            tmem_ld32(taddr + c * 32, a);
-            tmem_wait_ld();
+          uint32_t a[32];
+          tmem_ld32(taddr + c * 32, a);
+          tmem_wait_ld();
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              uint4 o;
-              uint32_t* ou = reinterpret_cast<uint32_t*>(&o);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(a[8 * v + 2 * i]),
-                                                               __uint_as_float(a[8 * v + 2 * i + 1]));
-                ou[i] = *reinterpret_cast<const uint32_t*>(&b);
-              }
-              *reinterpret_cast<uint4*>(dst + c * 32 + 8 * v) = o;
-            }
+          for (int i = 0; i < 16; ++i) {
+            const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
+            packed[c * 16 + i] = *reinterpret_cast<const uint32_t*>(&b);
           }
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));
+        __nv_bfloat16* dst = p.y + static_cast<size_t>(row) * p.d + w.nt * kBlockN;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (w.nt * kBlockN + c * 32 < p.d) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v)
+              *reinterpret_cast<uint4*>(dst + c * 32 + 8 * v) =
+                  make_uint4(packed[c * 16 + 4 * v], packed[c * 16 + 4 * v + 1], packed[c * 16 + 4 * v + 2], packed[c * 16 + 4 * v + 3]);
+          }
+        }
       }
     }
   }
@@ -341,19 +493,18 @@ ffn_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   }
 }
 
-template <int MODE>
-cudaError_t launch_ffn_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, int num_sms,
-                            cudaStream_t stream) {
-  cudaError_t e = cudaFuncSetAttribute(ffn_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(kGemmSmemBytes));
-  if (e != cudaSuccess) return e;
-  const int max_items = (p.M_cap / kTileM) * p.NT;
-  const int grid = max(1, min(num_sms, max_items));
-  ffn_gemm_kernel<MODE><<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(tmA, tmB, p);
-  return cudaGetLastError();
+size_t ffn_workspace_bytes(int M_cap) {
+  return ((2 * sizeof(int32_t) * static_cast<size_t>(M_cap / kTileM)) + 255) & ~static_cast<size_t>(255);
 }
 
-template cudaError_t launch_ffn_gemm<0>(const CUtensorMap&, const CUtensorMap&, const GemmParams&, int, cudaStream_t);
-template cudaError_t launch_ffn_gemm<1>(const CUtensorMap&, const CUtensorMap&, const GemmParams&, int, cudaStream_t);
+cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const FfnParams& p, int num_sms,
+                       cudaStream_t stream) {
+  cudaError_t e = cudaFuncSetAttribute(ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(kGemmSmemBytes));
+  if (e != cudaSuccess) return e;
+  const int grid = max(1, num_sms);   // one persistent CTA per SM; CTAs without work leave at once
+  ffn_kernel<<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(tmA1, tmA2, p);
+  return cudaGetLastError();
+}
 
 }  // namespace tempo

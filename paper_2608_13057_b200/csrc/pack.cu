@@ -1,11 +1,16 @@
 // One-time weight re-layout for the grouped GEMM kernels (off the hot path).
 //
 // Packed blob, in order (every section 1024-byte aligned):
-//   W13p   u8 [G][f/128][256][d]   per 128-column block jb of H: 128 gate rows then 128 up rows,
-//                                  so one 256-row B tile feeds both halves of SwiGLU
-//   W2p    u8 [G][d][f]            unchanged order
-//   SF13   u8 [G][f/128][J1][2][512]   UE8M0 scale atoms of W13p tiles (gate atom, up atom)
-//   SF2    u8 [G][ceil(d/256)][J2][2][512]   scale atoms of W2 tiles (two 128-row blocks per tile)
+//   W13t   u8 [G][f/128][d/128][256][128]   B tiles of the gate/up GEMM.  Tile (jb, kb) holds, for
+//          the 128-column block jb of H, 128 gate rows then 128 up rows (so one tile feeds both
+//          halves of SwiGLU) times the 128 K-bytes of block kb, stored exactly as the tensor core
+//          reads them from shared memory: rows of 128 bytes, 16-byte chunk c of row r at chunk
+//          position c ^ (r & 7) (the 128-byte swizzle).  A tile is one contiguous 32 KB read and
+//          the tiles of one (instance, jb) follow each other along K: the weight stream of the
+//          flat regime is sequential in HBM.
+//   W2t    u8 [G][ceil(d/256)][f/128][256][128]   same for the down GEMM (rows beyond d are zero)
+//   SF13   u8 [G][f/128][J1][2][512]   UE8M0 scale atoms of W13t tiles (gate atom, up atom)
+//   SF2    u8 [G][ceil(d/256)][J2][2][512]   scale atoms of W2t tiles (two 128-row blocks per tile)
 // An atom covers 128 rows x 4 K-blocks in the order the tensor core's scale copy consumes:
 // word (row%32)*4 + row/32 holds the 4 scale bytes of that row.  Weight scales are per 128x128
 // block, so all 128 rows of an atom carry the same word.  J = ceil((K/128)/4).
@@ -24,31 +29,35 @@ PackLayout pack_layout(int G, int d, int f) {
   L.NT2 = (d + 255) / 256;
   L.off_w13 = 0;
   L.off_w2 = align1k(L.off_w13 + static_cast<size_t>(G) * 2 * f * d);
-  L.off_sf13 = align1k(L.off_w2 + static_cast<size_t>(G) * d * f);
+  L.off_sf13 = align1k(L.off_w2 + static_cast<size_t>(G) * L.NT2 * 256 * f);
   L.off_sf2 = align1k(L.off_sf13 + static_cast<size_t>(G) * L.NT1 * L.J1 * 1024);
   L.total = align1k(L.off_sf2 + static_cast<size_t>(G) * L.NT2 * L.J2 * 1024);
   return L;
 }
 
-// rows of W13 are permuted: packed row (g, jb, half, r) <- source row (g, half*f + jb*128 + r)
-__global__ void pack_w13_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int G, int d, int f) {
-  const size_t chunks_per_row = d / 16;
-  const size_t total = static_cast<size_t>(G) * 2 * f * chunks_per_row;
+// One thread per 16-byte chunk of the packed tiles.  mode 0: W13 [G][2f][d] -> W13t; mode 1: W2
+// [G][d][f] -> W2t.  n_rows = source rows per instance, K = source row length.
+__global__ void pack_tiles_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, int G, int NT, int Kb,
+                                  int n_rows, int K, int mode) {
+  const size_t total = static_cast<size_t>(G) * NT * Kb * 256 * 8;
   for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < total;
        i += static_cast<size_t>(gridDim.x) * blockDim.x) {
-    const size_t prow = i / chunks_per_row, c = i % chunks_per_row;
-    const int g = static_cast<int>(prow / (2 * f));
-    const int within = static_cast<int>(prow % (2 * f));
-    const int jb = within / 256, half = (within % 256) / 128, r = within % 128;
-    const size_t srow = static_cast<size_t>(g) * 2 * f + static_cast<size_t>(half) * f + jb * 128 + r;
-    reinterpret_cast<uint4*>(dst)[prow * chunks_per_row + c] = reinterpret_cast<const uint4*>(src)[srow * chunks_per_row + c];
+    const int c = static_cast<int>(i & 7);
+    const int r = static_cast<int>((i >> 3) & 255);
+    size_t rest = i >> 11;
+    const int kb = static_cast<int>(rest % Kb);
+    rest /= Kb;
+    const int nt = static_cast<int>(rest % NT);
+    const int g = static_cast<int>(rest / NT);
+    int srow;
+    if (mode == 0) srow = (r < 128 ? 0 : n_rows / 2) + nt * 128 + (r & 127);
+    else srow = nt * 256 + r;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (srow < n_rows)
+      v = *reinterpret_cast<const uint4*>(src + (static_cast<size_t>(g) * n_rows + srow) * K + kb * 128 + c * 16);
+    const size_t tile = (static_cast<size_t>(g) * NT + nt) * Kb + kb;
+    *reinterpret_cast<uint4*>(dst + tile * 32768 + r * 128 + ((c ^ (r & 7)) << 4)) = v;
   }
-}
-
-__global__ void copy16_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t n) {
-  for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n;
-       i += static_cast<size_t>(gridDim.x) * blockDim.x)
-    dst[i] = src[i];
 }
 
 __device__ __forceinline__ uint32_t ue8m0_of(float s, uint32_t* bad) {
@@ -86,10 +95,8 @@ __global__ void pack_sf_kernel(const float* __restrict__ scales, uint8_t* __rest
 cudaError_t launch_pack(int G, int d, int f, const uint8_t* w13_q, const float* w13_s, const uint8_t* w2_q,
                         const float* w2_s, uint8_t* packed, uint32_t* status, cudaStream_t stream) {
   const PackLayout L = pack_layout(G, d, f);
-  pack_w13_kernel<<<1184, 256, 0, stream>>>(w13_q, packed + L.off_w13, G, d, f);
-  copy16_kernel<<<1184, 256, 0, stream>>>(reinterpret_cast<const uint4*>(w2_q),
-                                          reinterpret_cast<uint4*>(packed + L.off_w2),
-                                          static_cast<size_t>(G) * d * f / 16);
+  pack_tiles_kernel<<<2368, 256, 0, stream>>>(w13_q, packed + L.off_w13, G, L.NT1, d / 128, 2 * f, d, 0);
+  pack_tiles_kernel<<<2368, 256, 0, stream>>>(w2_q, packed + L.off_w2, G, L.NT2, f / 128, d, f, 1);
   pack_sf_kernel<<<G * L.NT1 * L.J1 * 2, 128, 0, stream>>>(w13_s, packed + L.off_sf13, G, 2 * f / 128, d / 128,
                                                           L.NT1, L.J1, 0, status);
   pack_sf_kernel<<<G * L.NT2 * L.J2 * 2, 128, 0, stream>>>(w2_s, packed + L.off_sf2, G, d / 128, f / 128, L.NT2,

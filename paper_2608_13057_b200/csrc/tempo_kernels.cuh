@@ -54,19 +54,33 @@ PackLayout pack_layout(int G, int d, int f);
 cudaError_t launch_pack(int G, int d, int f, const uint8_t* w13_q, const float* w13_s, const uint8_t* w2_q,
                         const float* w2_s, uint8_t* packed, uint32_t* status, cudaStream_t stream);
 
-struct GemmParams {
-  int Kb, JK, NT, rowsB, n_cols, G_max, M_cap, ld_out, J_out;
-  const uint8_t* sfa;
-  const uint8_t* sfb;
+// One of the two GEMMs of the FFN as the fused kernel sees it.
+struct GemmSide {
+  int Kb;        // K / 128
+  int JK;        // scale atoms along K = ceil(Kb / 4)
+  int NT;        // 256-column tiles per instance
+  const uint8_t* wt;     // packed B tiles, 32 KB each, [inst][nt][kb]
+  const uint8_t* sfa;    // scale atoms of the A operand
+  const uint8_t* sfb;    // scale atoms of the packed weights
+};
+
+struct FfnParams {
+  GemmSide side[2];      // 0: gate/up (A = a_q), 1: down (A = h_q)
+  int run_mask;          // bit 0: run the gate/up tiles, bit 1: run the down tiles
+  int G_max, M_cap;
+  int d, f;
+  int J_h;               // scale atoms along f of the H buffer
   const int32_t* inst_off;
   const int32_t* m_pad;
-  uint8_t* out_q;
-  uint8_t* out_sf;
-  __nv_bfloat16* out_y;
+  uint8_t* h_q;
+  uint8_t* h_sf;
+  __nv_bfloat16* y;
+  int32_t* ready;        // workspace: per M-tile, epilogue warps of finished gate/up tiles
+  int32_t* done;         // workspace: per M-tile, down tiles that have seen `ready` complete
   uint32_t* status;
 };
-template <int MODE>
-cudaError_t launch_ffn_gemm(const CUtensorMap& tmA, const CUtensorMap& tmB, const GemmParams& p, int num_sms,
-                            cudaStream_t stream);
+size_t ffn_workspace_bytes(int M_cap);
+cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const FfnParams& p, int num_sms,
+                       cudaStream_t stream);
 
 }  // namespace tempo

@@ -277,6 +277,17 @@ def test_sweep_points_sampled(B, G, N):
     _sampled_rows_check(B, wl, buf, rows_per_inst=2, n_tokens=8)
 
 
+def test_block_is_reproducible_run_to_run(B):
+    wl = W.config2()
+    buf = _run_block(B, wl)
+    first = (buf.h_q.clone(), buf.y.clone(), buf.out.clone())
+    for _ in range(5):
+        buf.run_block()
+    torch.cuda.synchronize()
+    assert torch.equal(first[0], buf.h_q) and torch.equal(first[1], buf.y) and torch.equal(first[2], buf.out)
+    assert int(buf.workspace.max().item()) == 0                  # the H-ready counters are left clean
+
+
 def test_pack_rejects_non_power_of_two_scales(B):
     wl = W.config1()
     buf = B.RankBuffers(wl.T, wl.k, wl.E, wl.G_max, wl.R_max, wl.d, wl.f)

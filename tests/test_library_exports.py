@@ -34,6 +34,7 @@ def test_host_only_entry_points_and_argument_errors():
     assert B.tempo_m_cap_bound(s) == 2048 + 20 * 128
     assert B.tempo_sf_bytes(256, 4096) == 2 * 8 * 512
     assert B.tempo_sf_bytes(128, 256) == 512            # 2 column blocks still take one atom
+    assert B.tempo_workspace_bytes(B.make_shape(256, 8, 128, 20, 2, 4096, 1536, 4608)) == 512
     s = B.make_shape(256, 8, 128, 20, 2, 4096, 1536, 4608)
     n = B.tempo_packed_weight_bytes(s)
     assert n >= 20 * 3 * 4096 * 1536 and n % 1024 == 0
