@@ -172,7 +172,7 @@ int tempo_permute_pad(const tempo_shape* s, const void* x_bf16, const int32_t* r
   if (!x_bf16 || !row_pair || !m_pad || !a_q || !a_sf || !status) return TEMPO_ERR_NULL;
   PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, m_pad,
                   static_cast<uint8_t*>(a_q), a_sf};
-  return launch_permute_pad(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+  return launch_permute_pad(p, sm_count(), static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
 
 int tempo_ffn_gate_up(const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,

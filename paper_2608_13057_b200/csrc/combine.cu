@@ -14,7 +14,9 @@ constexpr int kCombThreads = 256;
 __global__ void __launch_bounds__(kCombThreads) combine_kernel(const CombineParams p) {
   const int t = blockIdx.x;
   const int col = (blockIdx.y * kCombThreads + threadIdx.x) * 8;
+  pdl_trigger();
   if (col >= p.d) return;
+  pdl_wait();
   int nv = p.T;
   if (p.n_valid != nullptr) nv = max(0, min(*p.n_valid, p.T));
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
@@ -57,8 +59,7 @@ __global__ void __launch_bounds__(kCombThreads) combine_kernel(const CombinePara
 
 cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream) {
   const dim3 grid(p.T, (p.d / 8 + kCombThreads - 1) / kCombThreads);
-  combine_kernel<<<grid, kCombThreads, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(combine_kernel, grid, dim3(kCombThreads), 0, stream, p);
 }
 
 }  // namespace tempo

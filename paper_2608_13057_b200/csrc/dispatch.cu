@@ -1,4 +1,4 @@
-// Step 1: fused count + quota dispatch + padded grouped layout, one CTA, one launch.
+// Step 1: fused count + quota dispatch + padded grouped layout, one launch of one thread-block cluster.
 //
 // The paper's in-graph contract (Section 4.4): dispatch through the replica table fused with
 // count collection into a cumulative per-expert counter, CUDA-graph padding rows masked, rows
@@ -7,24 +7,52 @@
 // pairs of one expert are ranked by ascending pair index and cut into contiguous rank runs.
 //
 // Ranks come from scans, not from atomics, so the result is bit-reproducible:
-//   pass 1  every warp owns a contiguous range of pairs and builds its own histogram
-//           (__match_any_sync groups equal experts inside a 32-pair step);
-//   scan    per expert, an exclusive prefix over the 32 warp histograms gives each warp's base
-//           rank and the total n_e; the replica boundaries B_r follow from the quota row;
-//   pass 2  every warp walks its range again, rank = base + position among equal lanes.
+//   pass 1  the live pairs are cut into contiguous chunks, one per CTA of the cluster, and inside
+//           a CTA into one contiguous range per warp; every warp builds its own histogram
+//           (ballots over the id bits group equal experts inside a 32-pair step);
+//   scan    per expert, an exclusive prefix over the 32 warp histograms, then over the CTAs of the
+//           cluster (each CTA reads the others' totals through distributed shared memory), gives
+//           every warp's base rank and the total n_e; the replica boundaries B_r, the rows of
+//           each instance and the padded offsets follow from the quota row (every CTA computes
+//           them, CTA 0 writes them out);
+//   pass 2  every warp walks its range again, rank = base + position among equal lanes, and
+//           scatters pair -> row and row -> pair.
+// The cluster barriers are hardware barriers: nothing spins.
+#include <cooperative_groups.h>
+
 #include "tempo_kernels.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace tempo {
 
 constexpr int kDispThreads = 1024;
 constexpr int kDispWarps = kDispThreads / 32;
+constexpr int kKeep = 4;           // 32-pair steps of a warp whose ids stay in registers between the passes
+constexpr int kMaxCluster = 8;     // portable cluster size
+constexpr int kPairsPerCta = 4096; // pairs per CTA before another CTA joins the cluster
 
+// Lanes of the warp that hold the same expert id as this lane (e < 0: none).  One ballot per id
+// bit: a fixed, short latency, where __match_any_sync takes one round per distinct value.
+__device__ __forceinline__ uint32_t same_expert_mask(int e, int id_bits) {
+  uint32_t m = __ballot_sync(0xffffffffu, e >= 0);
+  for (int b = 0; b < id_bits; ++b) {
+    const uint32_t bal = __ballot_sync(0xffffffffu, (e >> b) & 1);
+    m &= ((e >> b) & 1) ? bal : ~bal;
+  }
+  return e >= 0 ? m : 0u;
+}
 
 __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const DispatchParams p) {
   extern __shared__ int32_t smem[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int NC = static_cast<int>(cluster.num_blocks());
+  const int cta = static_cast<int>(cluster.block_rank());
   const int E = p.E, R = p.R_max, G = p.G_max;
-  int32_t* hist = smem;                       // [kDispWarps][E]  warp histograms -> exclusive bases
-  int32_t* bnd = hist + kDispWarps * E;       // [E][R]           cumulative rank boundaries B_r
+  int32_t* hist = smem;                       // [kDispWarps][E]  warp histograms -> exclusive bases inside the CTA
+  int32_t* tot = hist + kDispWarps * E;       // [E]              this CTA's totals (read by the other CTAs)
+  int32_t* cbase = tot + E;                   // [E]              pairs of the expert in lower-ranked CTAs
+  int32_t* bnd = cbase + E;                   // [E][R]           cumulative rank boundaries B_r
   int32_t* owner = bnd + E * R;               // [G]              first (e,r) entry naming the slot
   int32_t* m_inst = owner + G;                // [G]              rows of each instance
   int32_t* off = m_inst + G;                  // [G+1]            padded offsets (not clamped)
@@ -34,10 +62,18 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
   __shared__ int32_t s_carry;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_trigger();
+  pdl_wait();
   int nv = p.T;
   if (p.n_valid != nullptr) nv = max(0, min(*p.n_valid, p.T));
   const int P = nv * p.k;                     // live pairs
   const int total_pairs = p.T * p.k;
+
+  // rows are scattered into after pass 1; every CTA pre-fills its share
+  for (int row = cta * kDispThreads + tid; row < p.M_cap; row += NC * kDispThreads) p.row_pair[row] = -1;
+  for (int q = P + cta * kDispThreads + tid; q < total_pairs; q += NC * kDispThreads) p.pair_row[q] = -1;
+  int id_bits = 0;
+  while ((1 << id_bits) < E) ++id_bits;
 
   // all table reads are issued up front, together with the first ids, so the kernel pays the
   // global-memory latency once
@@ -47,32 +83,42 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
   if (tid == 0) s_status = 0;
   __syncthreads();
 
-  // contiguous range of this warp, a multiple of 32 pairs long
-  const int per_warp = ((P + kDispWarps - 1) / kDispWarps + 31) & ~31;
-  const int w_begin = min(P, warp * per_warp), w_end = min(P, w_begin + per_warp);
+  // contiguous chunk of this CTA (a multiple of 1024 pairs) and range of this warp inside it
+  const int per_cta = (((P + NC - 1) / NC) + kDispThreads - 1) & ~(kDispThreads - 1);
+  const int c_begin = min(P, cta * per_cta), c_end = min(P, c_begin + per_cta);
+  const int per_warp = per_cta / kDispWarps;
+  const int w_begin = min(c_end, c_begin + warp * per_warp), w_end = min(c_end, w_begin + per_warp);
   uint32_t my_status = 0;
 
   // ---- pass 1: warp histograms -------------------------------------------------------------
-  for (int base = w_begin; base < w_end; base += 32) {
-    const int pidx = base + lane;
-    int e = -1;
-    if (pidx < w_end) {
-      e = __ldg(p.topk_ids + pidx);
-      if (e < 0 || e >= E) { my_status |= TEMPO_STATUS_BAD_ID; e = -1; }
+  int kept[kKeep];                            // ids of the first kKeep steps, reused by pass 2
+#pragma unroll
+  for (int i = 0; i < kKeep; ++i) kept[i] = -1;
+  {
+    int step = 0;
+    for (int base = w_begin; base < w_end; base += 32, ++step) {
+      const int pidx = base + lane;
+      int e = -1;
+      if (pidx < w_end) {
+        e = __ldg(p.topk_ids + pidx);
+        if (e < 0 || e >= E) { my_status |= TEMPO_STATUS_BAD_ID; e = -1; }
+      }
+#pragma unroll
+      for (int i = 0; i < kKeep; ++i) if (i == step) kept[i] = e;
+      const uint32_t same = same_expert_mask(e, id_bits);
+      if (e >= 0 && lane == __ffs(same) - 1) hist[warp * E + e] += __popc(same);
+      __syncwarp();
     }
-    const uint32_t same = __match_any_sync(0xffffffffu, e);
-    if (e >= 0 && lane == __ffs(same) - 1) hist[warp * E + e] += __popc(same);
-    __syncwarp();
   }
   // ---- which (e, r) owns each slot: the first entry in row-major order ----------------------
   for (int idx = tid; idx < E * R; idx += kDispThreads) {
     const int slot = rmap_s[idx];
     if (slot >= 0 && slot < G) atomicMin(&owner[slot], idx);
-    else if (slot != -1) my_status |= TEMPO_STATUS_BAD_TABLE;
+    else if (slot != -1 && cta == 0) my_status |= TEMPO_STATUS_BAD_TABLE;
   }
   __syncthreads();
 
-  // ---- per expert: totals, warp bases, replica boundaries -----------------------------------
+  // ---- per expert: warp bases inside the CTA, CTA total -------------------------------------
   for (int e = tid; e < E; e += kDispThreads) {
     int run = 0;
     for (int w = 0; w < kDispWarps; ++w) {
@@ -80,22 +126,37 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
       hist[w * E + e] = run;
       run += c;
     }
-    const int n_e = run;
-    p.counts[e] = n_e;
-    if (p.cum_counts != nullptr) atomicAdd(&p.cum_counts[e], static_cast<uint32_t>(n_e));
+    tot[e] = run;
+  }
+  cluster.sync();
+
+  // ---- per expert: base over lower CTAs, n_e, replica boundaries ------------------------------
+  for (int e = tid; e < E; e += kDispThreads) {
+    int n_e = 0, base = 0;
+    for (int c = 0; c < NC; ++c) {
+      const int v = c == cta ? tot[e] : *cluster.map_shared_rank(tot + e, c);
+      if (c < cta) base += v;
+      n_e += v;
+    }
+    cbase[e] = base;
+    if (cta == 0) {
+      p.counts[e] = n_e;
+      if (p.cum_counts != nullptr) atomicAdd(&p.cum_counts[e], static_cast<uint32_t>(n_e));
+    }
 
     unsigned long long S = 0;
-    uint32_t vmask = 0;
+    uint32_t vmask = 0, st = 0;
     for (int r = 0; r < R; ++r) {
       const int idx = e * R + r;
       const int slot = rmap_s[idx];
       const int x = quota_s[idx];
-      if (slot == -1) { if (x != 0) my_status |= TEMPO_STATUS_BAD_TABLE; continue; }
+      if (slot == -1) { if (x != 0) st |= TEMPO_STATUS_BAD_TABLE; continue; }
       if (slot < 0 || slot >= G) continue;                       // flagged above
-      if (owner[slot] != idx) { my_status |= TEMPO_STATUS_BAD_TABLE; continue; }
+      if (owner[slot] != idx) { st |= TEMPO_STATUS_BAD_TABLE; continue; }
       vmask |= 1u << r;
-      if (x < 0) my_status |= TEMPO_STATUS_BAD_TABLE; else S += static_cast<unsigned long long>(x);
+      if (x < 0) st |= TEMPO_STATUS_BAD_TABLE; else S += static_cast<unsigned long long>(x);
     }
+    if (cta == 0) my_status |= st;
     const bool uniform = (S == 0);
     if (uniform) S = __popc(vmask);
     unsigned long long C = 0;
@@ -104,7 +165,13 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
       const int idx = e * R + r;
       const bool valid = (vmask >> r) & 1u;
       if (valid) C += uniform ? 1ull : static_cast<unsigned long long>(max(quota_s[idx], 0));
-      const int B = S > 0 ? static_cast<int>(C * static_cast<unsigned long long>(n_e) / S) : 0;
+      int B = 0;
+      if (S > 0) {
+        if (C < 65536ull && S < 65536ull && n_e < 65536)
+          B = static_cast<int>(static_cast<uint32_t>(C) * static_cast<uint32_t>(n_e) / static_cast<uint32_t>(S));
+        else
+          B = static_cast<int>(C * static_cast<unsigned long long>(n_e) / S);
+      }
       bnd[idx] = B;
       if (valid) m_inst[rmap_s[idx]] = B - prev;
       prev = B;
@@ -136,42 +203,47 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
 
   const int M_pad_full = off[G];
   const int m_pad = min(M_pad_full, p.M_cap);
-  if (tid == 0) {
-    *p.m_pad = m_pad;
-    if (M_pad_full > p.M_cap) my_status |= TEMPO_STATUS_CAPACITY;
-  }
-  for (int i = tid; i <= G; i += kDispThreads) {
-    p.inst_off[i] = min(off[i], p.M_cap);
-    if (i < G) p.inst_count[i] = max(0, min(m_inst[i], p.M_cap - off[i]));
-  }
-  for (int row = tid; row < p.M_cap; row += kDispThreads) p.row_pair[row] = -1;
-  for (int q = P + tid; q < total_pairs; q += kDispThreads) p.pair_row[q] = -1;
-  for (int tau = tid; tau < p.M_cap / kTileM; tau += kDispThreads) {
-    const int row = tau * kTileM;
-    int inst = -1;
-    if (row < m_pad) {
-      int lo = 0, hi = G;                                        // first i with off[i+1] > row
-      while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (off[mid + 1] > row) hi = mid; else lo = mid + 1;
-      }
-      inst = lo;
+  if (cta == 0) {
+    if (tid == 0) {
+      *p.m_pad = m_pad;
+      if (M_pad_full > p.M_cap) my_status |= TEMPO_STATUS_CAPACITY;
     }
-    p.tile_inst[tau] = inst;
+    for (int i = tid; i <= G; i += kDispThreads) {
+      p.inst_off[i] = min(off[i], p.M_cap);
+      if (i < G) p.inst_count[i] = max(0, min(m_inst[i], p.M_cap - off[i]));
+    }
+    for (int tau = tid; tau < p.M_cap / kTileM; tau += kDispThreads) {
+      const int row = tau * kTileM;
+      int inst = -1;
+      if (row < m_pad) {
+        int lo = 0, hi = G;                                        // first i with off[i+1] > row
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (off[mid + 1] > row) hi = mid; else lo = mid + 1;
+        }
+        inst = lo;
+      }
+      p.tile_inst[tau] = inst;
+    }
   }
-  __syncthreads();   // row_pair is pre-filled before any thread scatters into it
+  // every CTA has pre-filled its share of row_pair, and nobody reads a neighbour's totals any more
+  cluster.sync();
 
   // ---- pass 2: stable ranks -> replica -> row -------------------------------------------------
-  for (int base = w_begin; base < w_end; base += 32) {
+  int step = 0;
+  for (int base = w_begin; base < w_end; base += 32, ++step) {
     const int pidx = base + lane;
     int e = -1;
-    if (pidx < w_end) {
+    if (step < kKeep) {
+#pragma unroll
+      for (int i = 0; i < kKeep; ++i) if (i == step) e = kept[i];
+    } else if (pidx < w_end) {
       e = __ldg(p.topk_ids + pidx);
       if (e < 0 || e >= E) e = -1;
     }
-    const uint32_t same = __match_any_sync(0xffffffffu, e);
+    const uint32_t same = same_expert_mask(e, id_bits);
     int j = 0;
-    if (e >= 0) j = hist[warp * E + e] + __popc(same & ((1u << lane) - 1u));
+    if (e >= 0) j = cbase[e] + hist[warp * E + e] + __popc(same & ((1u << lane) - 1u));
     __syncwarp();
     if (e >= 0 && lane == __ffs(same) - 1) hist[warp * E + e] += __popc(same);
     __syncwarp();
@@ -200,7 +272,8 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
 }
 
 size_t dispatch_smem_bytes(int E, int R, int G) {
-  return sizeof(int32_t) * (static_cast<size_t>(kDispWarps) * E + 3 * static_cast<size_t>(E) * R + 3 * static_cast<size_t>(G) + 1);
+  return sizeof(int32_t) * (static_cast<size_t>(kDispWarps + 2) * E + 3 * static_cast<size_t>(E) * R +
+                            3 * static_cast<size_t>(G) + 1);
 }
 
 cudaError_t launch_count_dispatch(const DispatchParams& p, cudaStream_t stream) {
@@ -208,8 +281,25 @@ cudaError_t launch_count_dispatch(const DispatchParams& p, cudaStream_t stream) 
   cudaError_t e = cudaFuncSetAttribute(count_dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  count_dispatch_kernel<<<1, kDispThreads, smem, stream>>>(p);
-  return cudaGetLastError();
+  const long long pairs = static_cast<long long>(p.T) * p.k;
+  int nc = 1;
+  while (nc < kMaxCluster && static_cast<long long>(nc) * kPairsPerCta < pairs) nc *= 2;
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(nc);
+  cfg.blockDim = dim3(kDispThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = nc;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, count_dispatch_kernel, p);
 }
 
 }  // namespace tempo

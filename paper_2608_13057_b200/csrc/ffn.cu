@@ -237,6 +237,24 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int G = p.G_max;
+  pdl_trigger();
+  // prologue that needs nothing from the previous kernel: barriers, tensor memory, descriptor fetch
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 2); mbar_init(smem_u32(&s_empty[s]), 1); }
+    mbar_init(smem_u32(&s_acc_full), 1);
+    mbar_init(smem_u32(&s_acc_empty), 4);
+    s_abort_storage = 0;
+    s_dep_storage = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA1)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA2)) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                 "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  pdl_wait();
   const int m_pad = max(0, min(*p.m_pad, p.M_cap)) & ~(kTileM - 1);
   const int m_tiles = m_pad / kTileM;
   const int n1 = (p.run_mask & 1) ? m_tiles * p.side[0].NT : 0;
@@ -245,20 +263,6 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   const int Kb1 = p.side[0].Kb, Kb2 = p.side[1].Kb;
 
   for (int i = tid; i <= G; i += kGemmThreads) s_toff[i] = max(0, min(p.inst_off[i], m_pad)) >> 7;
-  if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 2); mbar_init(smem_u32(&s_empty[s]), 1); }
-    mbar_init(smem_u32(&s_acc_full), 1);
-    mbar_init(smem_u32(&s_acc_empty), 4);
-    s_abort_storage = 0;
-    s_dep_storage = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
-                 "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -503,8 +507,7 @@ cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const F
                                        static_cast<int>(kGemmSmemBytes));
   if (e != cudaSuccess) return e;
   const int grid = max(1, num_sms);   // one persistent CTA per SM; CTAs without work leave at once
-  ffn_kernel<<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(tmA1, tmA2, p);
-  return cudaGetLastError();
+  return launch_pdl(ffn_kernel, dim3(grid), dim3(kGemmThreads), kGemmSmemBytes, stream, tmA1, tmA2, p);
 }
 
 }  // namespace tempo

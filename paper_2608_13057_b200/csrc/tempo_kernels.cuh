@@ -34,7 +34,7 @@ struct PermuteParams {
   uint8_t* a_q;
   uint8_t* a_sf;
 };
-cudaError_t launch_permute_pad(const PermuteParams& p, cudaStream_t stream);
+cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t stream);
 
 struct CombineParams {
   int T, k, d;
