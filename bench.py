@@ -4,8 +4,8 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3-uniform|...] [--impl reference]
     python bench.py --sweep            # cost-profile sweep (G, N grid) + max-affine fit -> n*
 
-One "step" is one pass of the whole hot path (count+dispatch, permute+quantise, gate/up GEMM + SwiGLU,
-down GEMM, combine) over one seeded synthetic routed batch, replayed as one CUDA graph.  Weight copies
+One "step" is one pass of the whole hot path (count+dispatch, permute+quantise, the fused gate/up + SwiGLU +
+down FFN kernel, combine) over one seeded synthetic routed batch, replayed as one CUDA graph.  Weight copies
 rotate through a pool larger than L2 so no step finds its weights cached (the paper's calibration
 protocol, Appendix B).  Rank 0 prints ONE JSON line.
 """
@@ -31,7 +31,7 @@ UNIT = "us_per_expert_block"
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_FP8_OVER_BF16 = 2.0             # dense fp8 peak = 2 x dense bf16 peak on this part
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the gate/up GEMM from the committed ncu
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel from the committed ncu
 # capture (profiles/), keyed by workload; None until a capture exists for that workload.
 NCU_TRAFFIC_BYTES = {}
 
@@ -249,8 +249,8 @@ def run_gpu(args):
 
     # ---- region B: the same steps launched call by call with events between the kernels -----------
     Kb = min(K, 200)
-    names = ["count_dispatch", "permute_pad", "ffn_gate_up", "ffn_down", "unpermute_combine"]
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(Kb)]
+    names = ["count_dispatch", "permute_pad", "grouped_ffn", "unpermute_combine"]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(Kb)]
     s = buf.shape
     torch.cuda._sleep(int(4e7))                        # keep the GPU busy so every launch is queued ahead
     for i in range(Kb):
@@ -262,12 +262,11 @@ def run_gpu(args):
         ev[i][1].record()
         B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status)
         ev[i][2].record()
-        B.tempo_ffn_gate_up(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.status)
+        B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y, buf.status,
+                            buf.workspace)
         ev[i][3].record()
-        B.tempo_ffn_down(s, buf.h_q, buf.h_sf, blob, buf.inst_off, buf.m_pad, buf.y, buf.status)
-        ev[i][4].record()
         B.tempo_unpermute_combine(s, buf.y, buf.pair_row, buf.topk_w, buf.n_valid, buf.out, buf.status)
-        ev[i][5].record()
+        ev[i][4].record()
     torch.cuda.synchronize()
     kern_us = {n: float(np.mean([ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(Kb)])) * 1e3
                for j, n in enumerate(names)}
@@ -314,19 +313,19 @@ def run_gpu(args):
     fp8_peak = peaks["bf16_tflops_sustained"] * NOMINAL_FP8_OVER_BF16
     tensor_time = st["padded_flops"] / (fp8_peak * 1e12) * 1e6
     bound = "hbm" if hbm_time >= tensor_time else "tensor"
-    # dominant kernel: the gate/up GEMM (2/3 of the weight bytes and of the FLOPs)
-    g1_us = kern_us["ffn_gate_up"]
+    # dominant kernel: the fused FFN kernel (both GEMMs of every activated instance in one launch)
+    ffn_us = kern_us["grouped_ffn"]
     if bound == "hbm":
-        alg = st["G_act"] * 2 * wl.d * wl.f                        # bytes: W13 of every activated instance
-        achieved = alg / (g1_us * 1e-6) / 1e9
+        alg = st["weight_bytes"]                                   # bytes: 3*d*f per activated instance
+        achieved = alg / (ffn_us * 1e-6) / 1e9
         roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
                     frac=achieved / peaks["hbm_gbs"], traffic=NCU_TRAFFIC_BYTES.get(args.workload))
     else:
-        alg = st["M_pad"] * 4 * wl.d * wl.f                        # flops: 2 * M_pad * 2f * d
-        achieved = alg / (g1_us * 1e-6) / 1e12
+        alg = st["padded_flops"]                                   # flops: 6*d*f per padded row
+        achieved = alg / (ffn_us * 1e-6) / 1e12
         roof = dict(bound="tensor", achieved=achieved, peak=fp8_peak, unit="TFLOP/s", frac=achieved / fp8_peak,
                     traffic=NCU_TRAFFIC_BYTES.get(args.workload))
-    roof.update(kernel="ffn_gemm_kernel<0> (gate/up + SwiGLU)", kernel_us=g1_us, peak_source=peaks["source"] +
+    roof.update(kernel="ffn_kernel (gate/up + SwiGLU + down, one launch)", kernel_us=ffn_us, peak_source=peaks["source"] +
                 (" HBM copy" if bound == "hbm" else " bf16 sustained x 2 (nominal fp8/bf16 ratio)"))
 
     out = {
@@ -340,8 +339,8 @@ def run_gpu(args):
         "block_us": us_step, "tokens_per_s": st["n_valid"] * world / (us_step * 1e-6),
         "block_roofline": {"weight_us": hbm_time, "padded_flop_us": tensor_time,
                            "frac": max(hbm_time, tensor_time) / us_step,
-                           "ffn_frac": max(hbm_time, tensor_time) / (kern_us["ffn_gate_up"] + kern_us["ffn_down"])},
-        "kernel_us": kern_us, "gpu_launches": 5 * K, "device_status": status,
+                           "ffn_frac": max(hbm_time, tensor_time) / kern_us["grouped_ffn"]},
+        "kernel_us": kern_us, "gpu_launches": 4 * K, "device_status": status,
         "roofline": roof, "clocks": clocks,
         "e2e": {"value": ms_e2e_max * 1e3 / units, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
     }
