@@ -161,6 +161,28 @@ int tempo_grouped_ffn(const tempo_shape* shape, const void* a_q, const uint8_t* 
                       uint32_t* status, void* workspace, void* stream);
 
 /*
+ * tempo_grouped_ffn without a caller-provided scratch buffer.  (The paper has no counterpart: this
+ * exists for the integration, not for the method.)  Some callers cannot allocate device memory at
+ * the point where they need the FFN: code that runs after the serving process has frozen its
+ * memory pool, a plug-in that is only handed the tensors of the layer, or a loop that must not
+ * risk the implicit device synchronisation cudaMalloc can cause.  For them the counters live in
+ * a 128 KB array built into the library image (one copy on every GPU that loads the library, held
+ * until the process exits).
+ *   - Same arguments, results and status bits as tempo_grouped_ffn, minus `workspace`.
+ *   - Limit: M_cap <= 2,097,152 rows (16384 tiles of 128).  A larger M_cap returns
+ *     TEMPO_ERR_UNSUPPORTED and launches nothing.
+ *   - Allocates nothing, ever.  The first call on each device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current); make that first call outside any stream
+ *     capture.  Every call enqueues a small cudaMemsetAsync of the counters before the kernel.
+ *   - All calls on a GPU share the one array: two calls that can overlap on the GPU (different
+ *     streams) race on it and give wrong results.  Serialise them, or use tempo_grouped_ffn with a
+ *     buffer per stream.
+ */
+int tempo_grouped_ffn_static(const tempo_shape* shape, const void* a_q, const uint8_t* a_sf, const void* packed,
+                             const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y_bf16,
+                             uint32_t* status, void* stream);
+
+/*
  * Step 4.  out[t,:] = sum_{s<k, pair_row[t*k+s] >= 0} topk_w[t,s] * y[pair_row[t*k+s], :], slots in
  * ascending order, fp32 accumulation, bf16 store.  Rows t >= n_valid and rows with no local pair are zero.
  *   in   y bf16 [M_cap, d], pair_row, topk_w f32 [T, k], n_valid (or NULL)     out  out bf16 [T, d]

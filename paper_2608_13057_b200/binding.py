@@ -21,7 +21,7 @@ EXPORTS = (
     "tempo_version", "tempo_status_string", "tempo_m_cap_bound", "tempo_sf_bytes", "tempo_workspace_bytes",
     "tempo_packed_weight_bytes",
     "tempo_pack_weights", "tempo_count_dispatch", "tempo_permute_pad", "tempo_ffn_gate_up", "tempo_ffn_down",
-    "tempo_grouped_ffn", "tempo_unpermute_combine",
+    "tempo_grouped_ffn", "tempo_grouped_ffn_static", "tempo_unpermute_combine",
 )
 
 
@@ -144,6 +144,17 @@ def tempo_grouped_ffn(shape, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf
                                   _ptr(h_q, torch.uint8), _ptr(h_sf, torch.uint8), _ptr(y_bf16, torch.bfloat16),
                                   _ptr(status, torch.int32), _ptr(workspace, torch.uint8), _stream()),
            "tempo_grouped_ffn")
+
+
+def tempo_grouped_ffn_static(shape, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status):
+    """tempo_grouped_ffn for callers that cannot provide scratch memory: the kernel's counters live in an
+    array built into the library (M_cap <= 2,097,152 rows).  Nothing is allocated.  Calls on one GPU must
+    not overlap; the first call on a device should come before any stream capture."""
+    _check(_lib.tempo_grouped_ffn_static(ctypes.byref(shape), _ptr(a_q, torch.uint8), _ptr(a_sf, torch.uint8),
+                                         _ptr(packed, torch.uint8), _ptr(inst_off, torch.int32),
+                                         _ptr(m_pad, torch.int32), _ptr(h_q, torch.uint8), _ptr(h_sf, torch.uint8),
+                                         _ptr(y_bf16, torch.bfloat16), _ptr(status, torch.int32), _stream()),
+           "tempo_grouped_ffn_static")
 
 
 def tempo_unpermute_combine(shape, y_bf16, pair_row, topk_w, n_valid, out_bf16, status):

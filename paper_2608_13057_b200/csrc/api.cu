@@ -90,6 +90,27 @@ static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, 
   return launch_ffn(tmA1, tmA2, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
 
+// ---- scratch for tempo_grouped_ffn_static ---------------------------------------------------------
+// The H-ready / down-seen counters of the fused FFN kernel, two int32 per 128-row tile, for callers
+// that cannot hand in a scratch buffer of their own.  Lives in every GPU that loads the library
+// (128 KB) until the process ends.  The name is a host-side handle here: the device address is
+// looked up once per device with cudaGetSymbolAddress and cached.
+constexpr int kStaticMaxTiles = 16384;                       // M_cap <= 128 * 16384 = 2,097,152 rows
+static __device__ __align__(256) int32_t g_ffn_scratch[2 * kStaticMaxTiles];
+constexpr int kMaxDevices = 64;
+static int32_t* g_ffn_scratch_addr[kMaxDevices] = {};
+
+static int32_t* static_scratch_for_current_device() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  if (g_ffn_scratch_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_ffn_scratch) != cudaSuccess || ptr == nullptr) return nullptr;
+    g_ffn_scratch_addr[dev] = static_cast<int32_t*>(ptr);
+  }
+  return g_ffn_scratch_addr[dev];
+}
+
 }  // namespace tempo
 
 using namespace tempo;
@@ -202,6 +223,23 @@ int tempo_grouped_ffn(const tempo_shape* s, const void* a_q, const uint8_t* a_sf
   if (!a_q || !a_sf || !packed || !inst_off || !m_pad || !h_q || !h_sf || !y_bf16 || !status || !workspace)
     return TEMPO_ERR_NULL;
   return launch_ffn_host(3, s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, workspace,
+                         static_cast<cudaStream_t>(stream));
+}
+
+int tempo_grouped_ffn_static(const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
+                             const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y_bf16,
+                             uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!a_q || !a_sf || !packed || !inst_off || !m_pad || !h_q || !h_sf || !y_bf16 || !status) return TEMPO_ERR_NULL;
+  if (s->M_cap / 128 > kStaticMaxTiles) return TEMPO_ERR_UNSUPPORTED;      // beyond the built-in scratch
+  int32_t* scratch = static_scratch_for_current_device();
+  if (scratch == nullptr) return TEMPO_ERR_CUDA;
+  // the array keeps whatever the last call left (normally zeros; not after a timed-out call): start clean
+  if (cudaMemsetAsync(scratch, 0, 2 * sizeof(int32_t) * static_cast<size_t>(s->M_cap / 128),
+                      static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return TEMPO_ERR_CUDA;
+  return launch_ffn_host(3, s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, scratch,
                          static_cast<cudaStream_t>(stream));
 }
 
