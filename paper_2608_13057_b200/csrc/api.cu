@@ -66,10 +66,13 @@ static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, 
   const uint8_t* blob = static_cast<const uint8_t*>(packed);
   const int sms = sm_count();
   if (sms <= 0) return TEMPO_ERR_CUDA;
-  CUtensorMap tmA1, tmA2;
+  CUtensorMap tmA1, tmA2, tmH, tmY;
   // a side that does not run still needs a well-formed map; point it at a buffer that exists
   if (!make_map(&tmA1, (run_mask & 1) ? a_q : h_q, s->M_cap, (run_mask & 1) ? s->d : s->f, 128)) return TEMPO_ERR_CUDA;
   if (!make_map(&tmA2, h_q, s->M_cap, s->f, 128)) return TEMPO_ERR_CUDA;
+  // stores: 32-row x 128-byte boxes of H (u8) and of Y (bf16 seen as bytes: 2d per row)
+  if (!make_map(&tmH, h_q, s->M_cap, s->f, 32)) return TEMPO_ERR_CUDA;
+  if (!make_map(&tmY, (run_mask & 2) ? y : h_q, s->M_cap, (run_mask & 2) ? 2ull * s->d : s->f, 32)) return TEMPO_ERR_CUDA;
   FfnParams p{};
   p.side[0] = GemmSide{s->d / 128, L.J1, L.NT1, blob + L.off_w13, a_sf, blob + L.off_sf13};
   p.side[1] = GemmSide{s->f / 128, L.J2, L.NT2, blob + L.off_w2, h_sf, blob + L.off_sf2};
@@ -87,7 +90,7 @@ static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, 
   p.ready = static_cast<int32_t*>(workspace);
   p.done = p.ready ? p.ready + s->M_cap / 128 : nullptr;
   p.status = status;
-  return launch_ffn(tmA1, tmA2, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+  return launch_ffn(tmA1, tmA2, tmH, tmY, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
 
 // ---- scratch for tempo_grouped_ffn_static ---------------------------------------------------------

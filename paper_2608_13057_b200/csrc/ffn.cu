@@ -23,7 +23,8 @@
 //   warp 1     MMA issuer: tcgen05.cp moves scale atoms into tensor memory, then four
 //              tcgen05.mma.kind::mxf8f6f4.block_scale (M128 N256 K32) per K-block accumulate in
 //              tensor memory; tcgen05.commit releases the stage / publishes the accumulator
-//   warps 2-5  epilogue: tcgen05.ld the accumulator (one row per thread), math, global stores
+//   warps 2-5  epilogue: tcgen05.ld the accumulator (one row per thread), math, swizzled staging in
+//              shared memory, TMA tensor stores
 // Scales are UE8M0 per 128 K-elements; the MMA takes one scale byte per row (A) and per column
 // (B) for each K=32 step, so the four steps of a K-block select the same byte (scale id kb % 4).
 //
@@ -49,7 +50,8 @@ constexpr int kTmemCols = 512;
 constexpr int kSfCol0 = 256;                              // scale slot s: A at 256+16s, B at 260+16s
 constexpr int kMaxSlots = 1024;
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
-constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 1024;
+constexpr int kStoreBytes = 32 * 128;                       // per-warp staging of a TMA store: 32 rows x 128 bytes
+constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 4 * kStoreBytes + 1024;
 
 
 // ---------------------------------------------------------------------------------------------
@@ -107,6 +109,19 @@ __device__ __forceinline__ void bulk_load_stream(uint32_t dst, const void* src, 
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar), "l"(policy)
       : "memory");
+}
+// TMA tensor store of a 32-row x 128-byte box from (swizzled) shared memory, bulk-group completion.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -221,7 +236,8 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 }
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
-ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2, const FfnParams p) {
+ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
+           const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmY, const FfnParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t s_full[kStages];
   __shared__ __align__(8) uint64_t s_empty[kStages];
@@ -248,6 +264,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA1)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA2)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmH)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
@@ -404,8 +422,14 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     }
   } else if (warp >= 2 && warp <= 5) {
     // ------------------------------- epilogue --------------------------------------------------
+    // Results leave through a per-warp 4 KB staging buffer (32 rows x 128 bytes, 128-byte swizzle so
+    // the 16-byte writes of a warp hit distinct banks) and one TMA tensor store per buffer: the
+    // global writes are full lines and do not compete with the producers' loads for the SM's
+    // load/store path, which row-per-thread 16-byte stores did.
     const int quad = warp & 3;                       // tensor-memory lanes this warp may read
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+    const uint32_t stage_buf = smem_base + kStages * kStageBytes + (warp - 2) * kStoreBytes;
+    const uint32_t my_line = stage_buf + lane * 128;
     uint32_t acc_phase = 0;
     TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
     int side, x;
@@ -437,7 +461,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));   // accumulator drained: the next tile may start
         const int eps = pow2_scale_exponent(amax);
         const float inv = pow2_neg(eps);
-        uint8_t* dst = p.h_q + static_cast<size_t>(row) * p.f + w.nt * 128;
+        if (lane == 0) bulk_wait_read();                      // the previous store has left the buffer
+        __syncwarp();
 #pragma unroll
         for (int v = 0; v < 8; ++v) {
           uint4 q;
@@ -445,13 +470,21 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
           q.y = cvt_e4m3x4(h[16 * v + 4] * inv, h[16 * v + 5] * inv, h[16 * v + 6] * inv, h[16 * v + 7] * inv);
           q.z = cvt_e4m3x4(h[16 * v + 8] * inv, h[16 * v + 9] * inv, h[16 * v + 10] * inv, h[16 * v + 11] * inv);
           q.w = cvt_e4m3x4(h[16 * v + 12] * inv, h[16 * v + 13] * inv, h[16 * v + 14] * inv, h[16 * v + 15] * inv);
-          *reinterpret_cast<uint4*>(dst + 16 * v) = q;
+          st_shared_v4(my_line + ((v ^ (lane & 7)) << 4), q);
         }
         p.h_sf[sf_index(row, w.nt, p.J_h)] = static_cast<uint8_t>(eps + 127);
-        if (fused) {                                  // publish this warp's 32 rows of the H block
-          __threadfence();
-          __syncwarp();
-          if (lane == 0) atomicAdd(p.ready + (w.row0 >> 7), 1);
+        fence_async_smem();
+        if (fused) __threadfence();                            // the scale byte, before the counter below
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&tmH, stage_buf, w.nt * 128, w.row0 + quad * 32);
+          bulk_commit();
+          if (fused) {                                         // publish this warp's 32 rows of the H block
+            bulk_wait_all();
+            asm volatile("fence.proxy.async;" ::: "memory");
+            __threadfence();
+            atomicAdd(p.ready + (w.row0 >> 7), 1);
+          }
         }
       } else {
         // drain the accumulator into packed bf16 registers first, release it, then store
@@ -470,18 +503,28 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));
-        __nv_bfloat16* dst = p.y + static_cast<size_t>(row) * p.d + w.nt * kBlockN;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          if (w.nt * kBlockN + c * 32 < p.d) {
+        for (int cg4 = 0; cg4 < 4; ++cg4) {                     // 64 columns = 128 bytes per row per store
+          if (w.nt * kBlockN + cg4 * 64 < p.d) {                // warp-uniform; the store clips at column d
+            if (lane == 0) bulk_wait_read();
+            __syncwarp();
 #pragma unroll
-            for (int v = 0; v < 4; ++v)
-              *reinterpret_cast<uint4*>(dst + c * 32 + 8 * v) =
-                  make_uint4(packed[c * 16 + 4 * v], packed[c * 16 + 4 * v + 1], packed[c * 16 + 4 * v + 2], packed[c * 16 + 4 * v + 3]);
+            for (int v = 0; v < 8; ++v)
+              st_shared_v4(my_line + ((v ^ (lane & 7)) << 4),
+                           make_uint4(packed[cg4 * 32 + 4 * v], packed[cg4 * 32 + 4 * v + 1], packed[cg4 * 32 + 4 * v + 2],
+                                      packed[cg4 * 32 + 4 * v + 3]));
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&tmY, stage_buf, (w.nt * kBlockN + cg4 * 64) * 2, w.row0 + quad * 32);
+              bulk_commit();
+            }
           }
         }
       }
     }
+    if (lane == 0) bulk_wait_all();                             // stores still read the staging buffer
+    __syncwarp();
   }
 
   tc_fence_before();
@@ -501,13 +544,13 @@ size_t ffn_workspace_bytes(int M_cap) {
   return ((2 * sizeof(int32_t) * static_cast<size_t>(M_cap / kTileM)) + 255) & ~static_cast<size_t>(255);
 }
 
-cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const FfnParams& p, int num_sms,
-                       cudaStream_t stream) {
+cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH, const CUtensorMap& tmY,
+                       const FfnParams& p, int num_sms, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(kGemmSmemBytes));
   if (e != cudaSuccess) return e;
   const int grid = max(1, num_sms);   // one persistent CTA per SM; CTAs without work leave at once
-  return launch_pdl(ffn_kernel, dim3(grid), dim3(kGemmThreads), kGemmSmemBytes, stream, tmA1, tmA2, p);
+  return launch_pdl(ffn_kernel, dim3(grid), dim3(kGemmThreads), kGemmSmemBytes, stream, tmA1, tmA2, tmH, tmY, p);
 }
 
 }  // namespace tempo

@@ -80,7 +80,7 @@ struct FfnParams {
   uint32_t* status;
 };
 size_t ffn_workspace_bytes(int M_cap);
-cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const FfnParams& p, int num_sms,
-                       cudaStream_t stream);
+cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH, const CUtensorMap& tmY,
+                       const FfnParams& p, int num_sms, cudaStream_t stream);
 
 }  // namespace tempo
