@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(kCombThreads) combine_kernel(const CombinePara
       }
 #pragma unroll
       for (int i = 0; i < 8; ++i)
-        v[i] = row[i] >= 0 ? __ldg(reinterpret_cast<const uint4*>(p.y + static_cast<size_t>(row[i]) * p.d + col))
+        v[i] = row[i] >= 0 ? __ldcs(reinterpret_cast<const uint4*>(p.y + static_cast<size_t>(row[i]) * p.d + col))
                            : make_uint4(0, 0, 0, 0);
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
@@ -54,7 +54,7 @@ __global__ void __launch_bounds__(kCombThreads) combine_kernel(const CombinePara
     const __nv_bfloat162 b = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
     ou[i] = *reinterpret_cast<const uint32_t*>(&b);
   }
-  *reinterpret_cast<uint4*>(p.out + static_cast<size_t>(t) * p.d + col) = o;
+  __stcs(reinterpret_cast<uint4*>(p.out + static_cast<size_t>(t) * p.d + col), o);
 }
 
 cudaError_t launch_combine(const CombineParams& p, cudaStream_t stream) {

@@ -9,8 +9,61 @@ namespace tempo {
 constexpr int kPermWarps = 8;
 
 
-// One warp per (row, 512-column chunk), grid-stride over the rows in use: a lane loads 32 bytes, the
-// 8 lanes of a 128-column block reduce its maximum, every lane stores 16 code bytes.
+// One warp per (row, 512-column chunk), grid-stride over the rows in use, two items per trip so the
+// gathers of both are in flight together: a lane loads 32 bytes, the 8 lanes of a 128-column block
+// reduce its maximum, every lane stores 16 code bytes.
+struct PermItem {
+  int row, col, pair;
+  bool live, in;
+  uint4 lo, hi;
+};
+
+__device__ __forceinline__ void perm_load(const PermuteParams& p, long long gw, long long n_items, int chunks, int lane,
+                                          PermItem& it) {
+  it.live = gw < n_items;
+  it.row = it.live ? static_cast<int>(gw / chunks) : 0;
+  it.col = it.live ? static_cast<int>(gw % chunks) * 512 + lane * 16 : 0;
+  it.in = it.live && it.col < p.d;                  // d is a multiple of 128, so 8-lane groups agree
+  it.pair = it.live ? __ldg(p.row_pair + it.row) : -1;
+  it.lo = make_uint4(0, 0, 0, 0);
+  it.hi = make_uint4(0, 0, 0, 0);
+}
+
+__device__ __forceinline__ void perm_gather(const PermuteParams& p, PermItem& it) {
+  if (it.in && it.pair >= 0) {
+    const __nv_bfloat16* src = p.x + static_cast<size_t>(it.pair / p.k) * p.d + it.col;
+    it.lo = __ldcs(reinterpret_cast<const uint4*>(src));
+    it.hi = __ldcs(reinterpret_cast<const uint4*>(src + 8));
+  }
+}
+
+__device__ __forceinline__ void perm_finish(const PermuteParams& p, const PermItem& it, int lane, int J) {
+  // padding rows come out as zero codes with scale 1 (all-zero block: eps = 0)
+  const uint32_t w[8] = {it.lo.x, it.lo.y, it.lo.z, it.lo.w, it.hi.x, it.hi.y, it.hi.z, it.hi.w};
+  float v[16];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+  float amax = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
+  if (!it.in) return;
+  const int eps = pow2_scale_exponent(amax);
+  const float inv = pow2_neg(eps);
+  uint4 q;
+  q.x = cvt_e4m3x4(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv);
+  q.y = cvt_e4m3x4(v[4] * inv, v[5] * inv, v[6] * inv, v[7] * inv);
+  q.z = cvt_e4m3x4(v[8] * inv, v[9] * inv, v[10] * inv, v[11] * inv);
+  q.w = cvt_e4m3x4(v[12] * inv, v[13] * inv, v[14] * inv, v[15] * inv);
+  __stcs(reinterpret_cast<uint4*>(p.a_q + static_cast<size_t>(it.row) * p.d + it.col), q);
+  if ((lane & 7) == 0) p.a_sf[sf_index(it.row, it.col >> 7, J)] = static_cast<uint8_t>(eps + 127);
+}
+
 __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_kernel(const PermuteParams p) {
   const int lane = threadIdx.x & 31;
   const int chunks = (p.d + 511) >> 9;
@@ -20,51 +73,14 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_kernel(const Perm
   const int m_pad = min(*p.m_pad, p.M_cap);
   const long long n_items = static_cast<long long>(m_pad) * chunks;
   const long long stride = static_cast<long long>(gridDim.x) * kPermWarps;
-  for (long long gw = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5); gw < n_items; gw += stride) {
-    const int row = static_cast<int>(gw / chunks);
-    const int col = static_cast<int>(gw % chunks) * 512 + lane * 16;
-    const int pair = p.row_pair[row];
-    const bool in = col < p.d;                      // d is a multiple of 128, so 8-lane groups agree
-    uint8_t* out = p.a_q + static_cast<size_t>(row) * p.d;
-
-    if (pair < 0) {                                 // padding row: zero codes, scale 1
-      if (in) {
-        *reinterpret_cast<uint4*>(out + col) = make_uint4(0, 0, 0, 0);
-        if ((lane & 7) == 0) p.a_sf[sf_index(row, col >> 7, J)] = 127;
-      }
-      continue;
-    }
-    float v[16];
-    if (in) {
-      const __nv_bfloat16* src = p.x + static_cast<size_t>(pair / p.k) * p.d + col;
-      const uint4 lo = __ldg(reinterpret_cast<const uint4*>(src));
-      const uint4 hi = __ldg(reinterpret_cast<const uint4*>(src + 8));
-      const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        v[2 * i] = __uint_as_float(w[i] << 16);
-        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-      }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 16; ++i) v[i] = 0.f;
-    }
-    float amax = 0.f;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
-    if (!in) continue;
-    const int eps = pow2_scale_exponent(amax);
-    const float inv = pow2_neg(eps);
-    uint4 q;
-    q.x = cvt_e4m3x4(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv);
-    q.y = cvt_e4m3x4(v[4] * inv, v[5] * inv, v[6] * inv, v[7] * inv);
-    q.z = cvt_e4m3x4(v[8] * inv, v[9] * inv, v[10] * inv, v[11] * inv);
-    q.w = cvt_e4m3x4(v[12] * inv, v[13] * inv, v[14] * inv, v[15] * inv);
-    *reinterpret_cast<uint4*>(out + col) = q;
-    if ((lane & 7) == 0) p.a_sf[sf_index(row, col >> 7, J)] = static_cast<uint8_t>(eps + 127);
+  for (long long gw = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5); gw < n_items; gw += 2 * stride) {
+    PermItem a, b;
+    perm_load(p, gw, n_items, chunks, lane, a);
+    perm_load(p, gw + stride, n_items, chunks, lane, b);
+    perm_gather(p, a);
+    perm_gather(p, b);
+    perm_finish(p, a, lane, J);
+    if (b.live) perm_finish(p, b, lane, J);
   }
 }
 
