@@ -288,6 +288,28 @@ def test_block_is_reproducible_run_to_run(B):
     assert int(buf.workspace.max().item()) == 0                  # the H-ready counters are left clean
 
 
+def test_bounded_wait_reports_timeout_and_the_context_stays_usable(B):
+    """Failure detection without a fault: the down tiles wait for H-ready counters that nothing will
+    complete (the workspace is poisoned on the host), the wait gives up after its one-second limit,
+    the kernel sets TEMPO_STATUS_TIMEOUT and returns; after re-zeroing the workspace the same buffers
+    produce the right result again."""
+    wl = W.config1()
+    buf = _run_block(B, wl)
+    good = buf.y.clone()
+    buf.workspace.view(torch.int32).fill_(-1000000)        # counters can never reach their target
+    buf.status.zero_()
+    B.tempo_grouped_ffn(buf.shape, buf.a_q, buf.a_sf, buf.packed, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
+                        buf.status, buf.workspace)
+    torch.cuda.synchronize()                                # returns after about one second
+    assert int(buf.status.item()) & B.STATUS_TIMEOUT
+    buf.workspace.zero_()
+    buf.status.zero_()
+    buf.run_block()
+    torch.cuda.synchronize()
+    assert int(buf.status.item()) == 0
+    assert torch.equal(buf.y[:int(buf.m_pad.item())], good[:int(buf.m_pad.item())])
+
+
 def test_pack_rejects_non_power_of_two_scales(B):
     wl = W.config1()
     buf = B.RankBuffers(wl.T, wl.k, wl.E, wl.G_max, wl.R_max, wl.d, wl.f)
