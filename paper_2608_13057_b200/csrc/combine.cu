@@ -7,11 +7,12 @@
 namespace tempo {
 
 constexpr int kCombThreads = 256;
+constexpr int kGroup = 4;   // slots whose gathers are in flight together
 
 // One thread per (token, 8 columns).  The k row indices and weights are read first, then all
-// gathers of a group of 8 slots are issued before any is consumed, so the thread pays the memory
+// gathers of a group of kGroup slots are issued before any is consumed, so the thread pays the memory
 // latency once per group instead of once per slot; the sum itself stays in slot order.
-__global__ void __launch_bounds__(kCombThreads) combine_kernel(const CombineParams p) {
+__global__ void __launch_bounds__(kCombThreads, 6) combine_kernel(const CombineParams p) {
   const int t = blockIdx.x;
   const int col = (blockIdx.y * kCombThreads + threadIdx.x) * 8;
   pdl_trigger();
@@ -21,22 +22,22 @@ __global__ void __launch_bounds__(kCombThreads) combine_kernel(const CombinePara
   if (p.n_valid != nullptr) nv = max(0, min(*p.n_valid, p.T));
   float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
   if (t < nv) {
-    for (int s0 = 0; s0 < p.k; s0 += 8) {
-      int row[8];
-      float w[8];
-      uint4 v[8];
+    for (int s0 = 0; s0 < p.k; s0 += kGroup) {
+      int row[kGroup];
+      float w[kGroup];
+      uint4 v[kGroup];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < kGroup; ++i) {
         const int s = s0 + i;
         row[i] = s < p.k ? __ldg(p.pair_row + t * p.k + s) : -1;
         w[i] = s < p.k ? __ldg(p.topk_w + t * p.k + s) : 0.f;
       }
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
+      for (int i = 0; i < kGroup; ++i)
         v[i] = row[i] >= 0 ? __ldcs(reinterpret_cast<const uint4*>(p.y + static_cast<size_t>(row[i]) * p.d + col))
                            : make_uint4(0, 0, 0, 0);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < kGroup; ++i) {
         if (row[i] < 0) continue;
         const uint32_t u[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
 #pragma unroll
