@@ -132,6 +132,27 @@ int tempo_count_dispatch(const tempo_shape* shape, const int32_t* topk_ids, cons
                          int32_t* row_pair, int32_t* tile_inst, int32_t* m_pad, uint32_t* status, void* stream);
 
 /*
+ * Step 1, sampled variant: the in-graph kernel as Section 4.4 describes it.  Same outputs and layout as
+ * tempo_count_dispatch, but the replica of each pair is drawn from its expert's row of a FLOAT share table:
+ *   table  f32 [E, R_max]  non-negative shares; only columns whose replica_map entry holds the expert
+ *          count; the row is renormalised at use; a row that sums to zero (or whose shares are all
+ *          invalid) falls back to uniform over the holders; negative / NaN / infinite shares, and shares
+ *          on a -1 column, count as zero and set TEMPO_STATUS_BAD_TABLE.  A torn or stale row therefore
+ *          costs a batch a stale or uniform split, never a wrong replica.
+ *   seed, layer  the draw for pair p is word 0 of Philox-4x32-10 with key (seed low, seed high) and counter
+ *          (p, 0, layer, 0): u = (word >> 8) * 2^-24; column = first holder r with u*S < C_r, S and the running
+ *          sums C_r accumulated in fp32 in column order (last holder if rounding leaves none).  The result is a
+ *          pure function of the arguments: replaying a graph with the same seed and layer repeats the dispatch;
+ *          advance `layer` (or the seed) per call for fresh draws.
+ * Rows of an instance are in ascending pair index.
+ */
+int tempo_count_dispatch_sampled(const tempo_shape* shape, const int32_t* topk_ids, const int32_t* n_valid,
+                                 const int32_t* replica_map, const float* table, uint64_t seed, uint32_t layer,
+                                 uint32_t* cum_counts, int32_t* counts, int32_t* inst_count, int32_t* inst_off,
+                                 int32_t* pair_row, int32_t* row_pair, int32_t* tile_inst, int32_t* m_pad,
+                                 uint32_t* status, void* stream);
+
+/*
  * Step 2.  a_q[row,:] = e4m3(x[row_pair[row]/k, :] / 2^eps) per 128-column block, eps the smallest
  * integer with max|block| <= 448 * 2^eps (0 for an all-zero block), round-to-nearest-even,
  * saturating; padding rows are zero codes with scale 1.  Rows >= m_pad are not written.

@@ -331,3 +331,137 @@ def expert_block(wl, M_cap=None, cum_counts=None):
         h_s = np.ones((M_cap, wl.f // QBLOCK), np.float32)
     out = combine(y, disp["pair_row"], wl.topk_w, wl.n_valid, wl.T, wl.k)
     return dict(disp, a_q=a_q, a_s=a_s, h_q=h_q, h_s=h_s, y=y, out=out)
+
+
+# ----------------------------------------------------------------------------------------
+# variant of step 1: probabilistic dispatch through a float share table (Section 4.4)
+# ----------------------------------------------------------------------------------------
+# The deployed kernel of the paper samples a replica per (token, slot) from a row of float shares,
+# renormalising the row at use and falling back to uniform over the replicas holding the expert when
+# the row sums to zero.  To make that reproducible both sides draw from the same counter-based
+# generator, Philox-4x32-10 (Salmon et al., "Parallel random numbers: as easy as 1, 2, 3", SC'11),
+# keyed by the seed and indexed by (pair index, layer): u = (word0 >> 8) * 2^-24.
+# Pins: the generator's published known-answer vectors; empirical replica frequencies against the
+# shares; the zero-sum and invalid-column rules; everything else as for the quota dispatch.
+
+_PHILOX_M0, _PHILOX_M1 = np.uint64(0xD2511F53), np.uint64(0xCD9E8D57)
+_PHILOX_W0, _PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32_10(counter, key):
+    """counter: uint32 [..., 4], key: uint32 [..., 2] -> uint32 [..., 4]."""
+    c = [np.asarray(counter)[..., i].astype(np.uint64) for i in range(4)]
+    k = [np.asarray(key)[..., i].astype(np.uint64) for i in range(2)]
+    mask = np.uint64(0xFFFFFFFF)
+    for _ in range(10):
+        p0 = _PHILOX_M0 * c[0]
+        p1 = _PHILOX_M1 * c[2]
+        hi0, lo0 = p0 >> np.uint64(32), p0 & mask
+        hi1, lo1 = p1 >> np.uint64(32), p1 & mask
+        c = [(hi1 ^ c[1] ^ k[0]) & mask, lo1, (hi0 ^ c[3] ^ k[1]) & mask, lo0]
+        k = [(k[0] + np.uint64(_PHILOX_W0)) & mask, (k[1] + np.uint64(_PHILOX_W1)) & mask]
+    return np.stack([v.astype(np.uint32) for v in c], axis=-1)
+
+
+def pair_uniform(seed, layer, n_pairs):
+    """u in [0,1) for pairs 0..n_pairs-1, fp32 with 24 random bits."""
+    ctr = np.zeros((n_pairs, 4), dtype=np.uint32)
+    ctr[:, 0] = np.arange(n_pairs, dtype=np.uint64).astype(np.uint32)
+    ctr[:, 2] = np.uint32(layer)
+    key = np.array([seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF], dtype=np.uint32)
+    w0 = philox4x32_10(ctr, np.broadcast_to(key, (n_pairs, 2)))[:, 0]
+    return ((w0 >> np.uint32(8)).astype(np.float32) * np.float32(2.0 ** -24)).astype(np.float32)
+
+
+def count_dispatch_sampled(topk_ids, n_valid, replica_map, table, seed, layer, G_max, M_cap, cum_counts=None):
+    """Like count_dispatch, but the replica of each pair is sampled from table[e, :] (float shares)."""
+    ids = np.asarray(topk_ids, dtype=np.int64)
+    T, k = ids.shape
+    rmap = np.asarray(replica_map)
+    tab = np.asarray(table, dtype=np.float32)
+    E, R = rmap.shape
+    n_valid = max(0, min(int(n_valid), T))
+    status = 0
+
+    # which columns hold the expert (same ownership rule as the quota variant), cleaned shares
+    claimed: set = set()
+    valid = np.zeros((E, R), dtype=bool)
+    q = np.zeros((E, R), dtype=np.float32)
+    for e in range(E):
+        for r in range(R):
+            s, x = int(rmap[e, r]), tab[e, r]
+            if s == -1:
+                if x != 0 or np.isnan(x):
+                    status |= STATUS_BAD_TABLE
+                continue
+            if s < 0 or s >= G_max or s in claimed:
+                status |= STATUS_BAD_TABLE
+                continue
+            claimed.add(s)
+            valid[e, r] = True
+            if not np.isfinite(x) or x < 0:
+                status |= STATUS_BAD_TABLE
+                x = np.float32(0.0)
+            q[e, r] = x
+
+    u = pair_uniform(seed, layer, T * k)
+    seen = [0] * E
+    slot_of = [-1] * (T * k)
+    m = [0] * G_max
+    pos = [0] * (T * k)
+    for p in range(n_valid * k):
+        e = int(ids[p // k, p % k])
+        if e < 0 or e >= E:
+            status |= STATUS_BAD_ID
+            continue
+        seen[e] += 1
+        cols = [r for r in range(R) if valid[e, r]]
+        if not cols:
+            continue                                      # expert not on this rank
+        S = np.float32(0.0)
+        for r in cols:
+            S = np.float32(S + q[e, r])                   # fp32 running sum in column order
+        w = q[e] if S > 0 else valid[e].astype(np.float32)   # zero-sum row: uniform over holders
+        if not S > 0:
+            S = np.float32(len(cols))
+        thr = np.float32(u[p] * S)                        # one fp32 multiply, compared with fp32 running sums
+        C = np.float32(0.0)
+        pick = cols[-1]
+        for r in cols:
+            C = np.float32(C + w[r])
+            if thr < C:
+                pick = r
+                break
+        i = int(rmap[e, pick])
+        slot_of[p] = i
+        pos[p] = m[i]
+        m[i] += 1
+    counts = np.array(seen, dtype=np.int32)
+
+    off = [0] * (G_max + 1)
+    for i in range(G_max):
+        off[i + 1] = off[i] + TILE_M * ((m[i] + TILE_M - 1) // TILE_M)
+    M_pad = off[G_max]
+    if M_pad > M_cap:
+        status |= STATUS_CAPACITY
+    pair_row = np.full(T * k, -1, dtype=np.int32)
+    row_pair = np.full(M_cap, -1, dtype=np.int32)
+    for p in range(n_valid * k):
+        if slot_of[p] >= 0:
+            row = off[slot_of[p]] + pos[p]
+            if row < M_cap:
+                pair_row[p] = row
+                row_pair[row] = p
+    inst_off = np.minimum(np.array(off, dtype=np.int64), M_cap).astype(np.int32)
+    inst_count = np.array([max(0, min(m[i], M_cap - off[i])) for i in range(G_max)], dtype=np.int32)
+    m_pad = min(M_pad, M_cap)
+    tile_inst = np.full(M_cap // TILE_M, -1, dtype=np.int32)
+    for i in range(G_max):
+        for tau in range(inst_off[i] // TILE_M, inst_off[i + 1] // TILE_M):
+            tile_inst[tau] = i
+    out = dict(counts=counts, inst_count=inst_count, inst_off=inst_off, pair_row=pair_row, row_pair=row_pair,
+               tile_inst=tile_inst, m_pad=np.int32(m_pad), status=np.uint32(status), slot_of=np.array(slot_of))
+    if cum_counts is not None:
+        out["cum_counts"] = ((np.asarray(cum_counts, dtype=np.uint64) + counts.astype(np.uint64))
+                             % (1 << 32)).astype(np.uint32)
+    return out

@@ -20,7 +20,7 @@ STATUS_BAD_ID, STATUS_BAD_TABLE, STATUS_CAPACITY, STATUS_TIMEOUT, STATUS_BAD_SCA
 EXPORTS = (
     "tempo_version", "tempo_status_string", "tempo_m_cap_bound", "tempo_sf_bytes", "tempo_workspace_bytes",
     "tempo_packed_weight_bytes",
-    "tempo_pack_weights", "tempo_count_dispatch", "tempo_permute_pad", "tempo_ffn_gate_up", "tempo_ffn_down",
+    "tempo_pack_weights", "tempo_count_dispatch", "tempo_count_dispatch_sampled", "tempo_permute_pad", "tempo_ffn_gate_up", "tempo_ffn_down",
     "tempo_grouped_ffn", "tempo_grouped_ffn_static", "tempo_unpermute_combine",
 )
 
@@ -117,6 +117,18 @@ def tempo_count_dispatch(shape, topk_ids, n_valid, replica_map, quota, cum_count
                                      _ptr(counts, i32), _ptr(inst_count, i32), _ptr(inst_off, i32),
                                      _ptr(pair_row, i32), _ptr(row_pair, i32), _ptr(tile_inst, i32),
                                      _ptr(m_pad, i32), _ptr(status, i32), _stream()), "tempo_count_dispatch")
+
+
+def tempo_count_dispatch_sampled(shape, topk_ids, n_valid, replica_map, table, seed, layer, cum_counts, counts,
+                                 inst_count, inst_off, pair_row, row_pair, tile_inst, m_pad, status):
+    i32 = torch.int32
+    _check(_lib.tempo_count_dispatch_sampled(ctypes.byref(shape), _ptr(topk_ids, i32), _ptr(n_valid, i32),
+                                             _ptr(replica_map, i32), _ptr(table, torch.float32),
+                                             ctypes.c_uint64(int(seed)), ctypes.c_uint32(int(layer)),
+                                             _ptr(cum_counts, i32), _ptr(counts, i32), _ptr(inst_count, i32),
+                                             _ptr(inst_off, i32), _ptr(pair_row, i32), _ptr(row_pair, i32),
+                                             _ptr(tile_inst, i32), _ptr(m_pad, i32), _ptr(status, i32), _stream()),
+           "tempo_count_dispatch_sampled")
 
 
 def tempo_permute_pad(shape, x_bf16, row_pair, m_pad, a_q, a_sf, status):

@@ -19,6 +19,7 @@ static int check_shape(const tempo_shape* s) {
   if (static_cast<long long>(s->T) * s->k > 0x7fff0000ll || static_cast<long long>(s->M_cap) > 0x7fff0000ll)
     return TEMPO_ERR_UNSUPPORTED;
   if (dispatch_smem_bytes(s->E, s->R_max, s->G_max) > 220 * 1024) return TEMPO_ERR_UNSUPPORTED;
+  if (dispatch_sampled_smem_bytes(s->E, s->R_max, s->G_max) > 220 * 1024) return TEMPO_ERR_UNSUPPORTED;
   return TEMPO_OK;
 }
 
@@ -187,6 +188,22 @@ int tempo_count_dispatch(const tempo_shape* s, const int32_t* topk_ids, const in
   DispatchParams p{s->T, s->k, s->E, s->G_max, s->R_max, s->M_cap, topk_ids, n_valid, replica_map, quota,
                    cum_counts, counts, inst_count, inst_off, pair_row, row_pair, tile_inst, m_pad, status};
   return launch_count_dispatch(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+int tempo_count_dispatch_sampled(const tempo_shape* s, const int32_t* topk_ids, const int32_t* n_valid,
+                                 const int32_t* replica_map, const float* table, uint64_t seed, uint32_t layer,
+                                 uint32_t* cum_counts, int32_t* counts, int32_t* inst_count, int32_t* inst_off,
+                                 int32_t* pair_row, int32_t* row_pair, int32_t* tile_inst, int32_t* m_pad,
+                                 uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!topk_ids || !replica_map || !table || !counts || !inst_count || !inst_off || !pair_row || !row_pair ||
+      !tile_inst || !m_pad || !status)
+    return TEMPO_ERR_NULL;
+  SampledParams p{s->T, s->k, s->E, s->G_max, s->R_max, s->M_cap, topk_ids, n_valid, replica_map, table,
+                  static_cast<unsigned long long>(seed), layer, cum_counts, counts, inst_count, inst_off, pair_row,
+                  row_pair, tile_inst, m_pad, status};
+  return launch_count_dispatch_sampled(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
 
 int tempo_permute_pad(const tempo_shape* s, const void* x_bf16, const int32_t* row_pair, const int32_t* m_pad,

@@ -20,28 +20,11 @@
 // The cluster barriers are hardware barriers: nothing spins.
 #include <cooperative_groups.h>
 
-#include "tempo_kernels.cuh"
+#include "dispatch_common.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace tempo {
-
-constexpr int kDispThreads = 1024;
-constexpr int kDispWarps = kDispThreads / 32;
-constexpr int kKeep = 4;           // 32-pair steps of a warp whose ids stay in registers between the passes
-constexpr int kMaxCluster = 8;     // portable cluster size
-constexpr int kPairsPerCta = 4096; // pairs per CTA before another CTA joins the cluster
-
-// Lanes of the warp that hold the same expert id as this lane (e < 0: none).  One ballot per id
-// bit: a fixed, short latency, where __match_any_sync takes one round per distinct value.
-__device__ __forceinline__ uint32_t same_expert_mask(int e, int id_bits) {
-  uint32_t m = __ballot_sync(0xffffffffu, e >= 0);
-  for (int b = 0; b < id_bits; ++b) {
-    const uint32_t bal = __ballot_sync(0xffffffffu, (e >> b) & 1);
-    m &= ((e >> b) & 1) ? bal : ~bal;
-  }
-  return e >= 0 ? m : 0u;
-}
 
 __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const DispatchParams p) {
   extern __shared__ int32_t smem[];
@@ -278,28 +261,7 @@ size_t dispatch_smem_bytes(int E, int R, int G) {
 
 cudaError_t launch_count_dispatch(const DispatchParams& p, cudaStream_t stream) {
   const size_t smem = dispatch_smem_bytes(p.E, p.R_max, p.G_max);
-  cudaError_t e = cudaFuncSetAttribute(count_dispatch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
-  if (e != cudaSuccess) return e;
-  const long long pairs = static_cast<long long>(p.T) * p.k;
-  int nc = 1;
-  while (nc < kMaxCluster && static_cast<long long>(nc) * kPairsPerCta < pairs) nc *= 2;
-
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(nc);
-  cfg.blockDim = dim3(kDispThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  attr[1].id = cudaLaunchAttributeClusterDimension;
-  attr[1].val.clusterDim.x = nc;
-  attr[1].val.clusterDim.y = 1;
-  attr[1].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, count_dispatch_kernel, p);
+  return launch_dispatch_cluster(count_dispatch_kernel, p, static_cast<long long>(p.T) * p.k, smem, stream);
 }
 
 }  // namespace tempo

@@ -24,6 +24,27 @@ struct DispatchParams {
   uint32_t* status;
 };
 size_t dispatch_smem_bytes(int E, int R, int G);
+
+struct SampledParams {
+  int T, k, E, G_max, R_max, M_cap;
+  const int32_t* topk_ids;
+  const int32_t* n_valid;
+  const int32_t* replica_map;
+  const float* table;
+  unsigned long long seed;
+  uint32_t layer;
+  uint32_t* cum_counts;
+  int32_t* counts;
+  int32_t* inst_count;
+  int32_t* inst_off;
+  int32_t* pair_row;
+  int32_t* row_pair;
+  int32_t* tile_inst;
+  int32_t* m_pad;
+  uint32_t* status;
+};
+size_t dispatch_sampled_smem_bytes(int E, int R, int G);
+cudaError_t launch_count_dispatch_sampled(const SampledParams& p, cudaStream_t stream);
 cudaError_t launch_count_dispatch(const DispatchParams& p, cudaStream_t stream);
 
 struct PermuteParams {

@@ -105,6 +105,38 @@ def test_count_dispatch_bit_exact(B, wl):
     _assert_dispatch_equal(got, ref)
 
 
+def _sampled_cases():
+    g = np.random.default_rng(11)
+    for wl in (W.config1(), W.config2(), W.config2(n_valid=200), W.config3("uniform"), W.config4(with_x=False),
+               W.config5_point(64, 1024, with_x=False), W.random_small(500, T=200, E=37, k=3), W.random_small(501, T=9, n_valid=0)):
+        table = (g.random(wl.replica_map.shape) * (g.random(wl.replica_map.shape) < 0.8)).astype(np.float32)
+        yield wl, table
+    wl = W.random_small(502, T=300, E=6, k=2)
+    table = g.random(wl.replica_map.shape).astype(np.float32)
+    table[0, 0], table[1, 0], table[2, :] = np.nan, -1.0, 0.0          # bad shares, a zero-sum row
+    table[wl.replica_map < 0] = 2.0                                    # shares on columns that hold nothing
+    yield wl, table
+
+
+@pytest.mark.parametrize("wl,table", list(_sampled_cases()), ids=lambda v: getattr(v, "name", None))
+def test_count_dispatch_sampled_bit_exact(B, wl, table):
+    buf = B.RankBuffers(wl.T, wl.k, wl.E, wl.G_max, wl.R_max, 128, 128)
+    buf.topk_ids.copy_(torch.from_numpy(wl.topk_ids))
+    buf.n_valid.fill_(int(wl.n_valid))
+    buf.replica_map.copy_(torch.from_numpy(wl.replica_map))
+    cum = np.full(wl.E, 2 ** 32 - 5, np.uint32)
+    buf.cum_counts.copy_(torch.from_numpy(cum.view(np.int32)))
+    t_dev = torch.from_numpy(table).cuda()
+    seed, layer = 0x9E3779B97F4A7C15, 17
+    B.tempo_count_dispatch_sampled(buf.shape, buf.topk_ids, buf.n_valid, buf.replica_map, t_dev, seed, layer,
+                                   buf.cum_counts, buf.counts, buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair,
+                                   buf.tile_inst, buf.m_pad, buf.status)
+    torch.cuda.synchronize()
+    ref = O.count_dispatch_sampled(wl.topk_ids, wl.n_valid, wl.replica_map, table, seed, layer, wl.G_max, buf.M_cap,
+                                   cum_counts=cum)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+
+
 def test_count_dispatch_capacity_overflow(B):
     ids = (np.arange(600, dtype=np.int32) % 2).reshape(600, 1)
     wl = _table_case(ids, 600, [[0], [1]], [[300], [300]], 2, "capacity")
