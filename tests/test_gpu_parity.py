@@ -320,6 +320,35 @@ def test_block_is_reproducible_run_to_run(B):
     assert int(buf.workspace.max().item()) == 0                  # the H-ready counters are left clean
 
 
+def test_graph_replay_matches_eager_launches(B):
+    """The launch configuration bench.py times: the four calls captured in one CUDA graph and replayed,
+    with the weights coming from a rotated copy.  Replays must reproduce the eager result bit for bit."""
+    wl = W.config2()
+    buf = _run_block(B, wl)
+    eager = (buf.pair_row.clone(), buf.a_q.clone(), buf.h_q.clone(), buf.y.clone(), buf.out.clone())
+    other = buf.packed.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        buf.run_block(packed=other)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        buf.run_block(packed=other)
+    for t in (buf.pair_row, buf.a_q, buf.h_q, buf.y, buf.out):
+        t.zero_()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(eager, (buf.pair_row, buf.a_q, buf.h_q, buf.y, buf.out)):
+        assert torch.equal(a, b)
+    assert int(buf.status.item()) == 0
+    ref = O.expert_block(wl, M_cap=buf.M_cap)
+    mx, mean = _err(to_np(buf.out), ref["out"])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL
+
+
 def test_bounded_wait_reports_timeout_and_the_context_stays_usable(B):
     """Failure detection without a fault: the down tiles wait for H-ready counters that nothing will
     complete (the workspace is poisoned on the host), the wait gives up after its one-second limit,
