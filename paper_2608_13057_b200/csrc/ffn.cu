@@ -14,17 +14,19 @@
 // so HBM keeps streaming.  The counters clean themselves: the last down tile of an M-tile to see
 // the counter complete puts it back to zero.
 //
-// Per CTA (one per SM, 256 threads):
+// Per CTA (one per SM, 384 threads):
 //   warp 0     weight producer: per K-block one contiguous 32 KB bulk copy of a pre-swizzled
 //              packed B tile (+ two 512-byte scale atoms every 4th K-block) into a 4-stage ring
-//   warp 6     activation producer: per K-block a 128x128 A tile (TMA tensor copy, 128-byte
+//   warp 2     activation producer: per K-block a 128x128 A tile (TMA tensor copy, 128-byte
 //              swizzle) (+ one scale atom every 4th K-block); waits for H where needed
-//   warp 7     dependency scout: runs ahead of warp 6 through the down tiles, watches the H counters
+//   warp 3     dependency scout: runs ahead of warp 2 through the down tiles, watches the H counters
 //   warp 1     MMA issuer: tcgen05.cp moves scale atoms into tensor memory, then four
 //              tcgen05.mma.kind::mxf8f6f4.block_scale (M128 N256 K32) per K-block accumulate in
 //              tensor memory; tcgen05.commit releases the stage / publishes the accumulator
-//   warps 2-5  epilogue: tcgen05.ld the accumulator (one row per thread), math, swizzled staging in
-//              shared memory, TMA tensor stores
+//   warps 4-11 epilogue, two warps per tensor-memory lane quadrant, each taking half of a row's
+//              columns: tcgen05.ld the raw accumulator into registers and hand tensor memory back
+//              to the MMA issuer at once, then the math (the pair shares the row maximum through
+//              shared memory), swizzled staging in shared memory, TMA tensor stores
 // Scales are UE8M0 per 128 K-elements; the MMA takes one scale byte per row (A) and per column
 // (B) for each K=32 step, so the four steps of a K-block select the same byte (scale id kb % 4).
 //
@@ -44,7 +46,8 @@ constexpr int kBBytes = kBlockN * kBlockK;                // 32 KB
 constexpr int kSfaBytes = 512;
 constexpr int kSfbBytes = 1024;
 constexpr int kStageBytes = kABytes + kBBytes + 2048;     // 51200, a multiple of 1024
-constexpr int kGemmThreads = 256;
+constexpr int kGemmThreads = 384;
+constexpr int kEpiWarp0 = 4;                               // first of the 8 epilogue warps
 constexpr int kTileOverhead = 5;                          // per-tile fixed cost in K-block steps (ramp + epilogue)
 constexpr int kTmemCols = 512;
 constexpr int kSfCol0 = 256;                              // scale slot s: A at 256+16s, B at 260+16s
@@ -153,6 +156,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Named barrier of two warps (64 threads).
+__device__ __forceinline__ void pair_sync(int id) { asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory"); }
+// Compiler-level pin: the 32 values are treated as produced here, so nothing computed from them
+// can be scheduled above this point.
+__device__ __forceinline__ void pin32(uint32_t (&r)[32]) {
+#pragma unroll
+  for (int i = 0; i < 32; i += 8)
+    asm volatile("" : "+r"(r[i]), "+r"(r[i + 1]), "+r"(r[i + 2]), "+r"(r[i + 3]), "+r"(r[i + 4]), "+r"(r[i + 5]),
+                      "+r"(r[i + 6]), "+r"(r[i + 7])
+                 :: "memory");
+}
 
 // Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows of 128 bytes, groups of
 // 8 rows 1024 bytes apart (stride byte offset), descriptor version 1.
@@ -247,6 +261,8 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   __shared__ int s_abort_storage;
   __shared__ int s_dep_storage;
   __shared__ int s_toff[kMaxSlots + 1];
+  __shared__ float s_amax[2][2][kTileM];   // [tile parity][column half][row]: row maxima of the two half-row warps
+  __shared__ int s_ok[2][4][2];             // [tile parity][quadrant][column half]: that warp's wait succeeded
   volatile int* s_abort = &s_abort_storage;
   volatile int* s_dep = &s_dep_storage;   // down tiles of this CTA whose H rows are known complete
 
@@ -258,7 +274,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 2); mbar_init(smem_u32(&s_empty[s]), 1); }
     mbar_init(smem_u32(&s_acc_full), 1);
-    mbar_init(smem_u32(&s_acc_empty), 4);
+    mbar_init(smem_u32(&s_acc_empty), 8);
     s_abort_storage = 0;
     s_dep_storage = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -312,7 +328,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         }
       }
     }
-  } else if (warp == 6) {
+  } else if (warp == 2) {
     // ------------------------------- activation producer --------------------------------------
     if (lane == 0) {
       uint32_t stage = 0, phase = 0;
@@ -326,7 +342,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         const uint8_t* sfa_src = gs.sfa + static_cast<size_t>(w.row0 >> 7) * gs.JK * kSfaBytes;
         const CUtensorMap* tm = side == 0 ? &tmA1 : &tmA2;
         if (side == 1 && fused) {
-          // wait until the scout (warp 7) has seen every H block of these 128 rows complete
+          // wait until the scout (warp 3) has seen every H block of these 128 rows complete
           ++n_down;
           unsigned long long t0 = 0;
           for (uint32_t spin = 0; *s_dep < n_down; ++spin) {
@@ -353,7 +369,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         }
       }
     }
-  } else if (warp == 7) {
+  } else if (warp == 3) {
     // ------------------------------- dependency scout -----------------------------------------
     // Runs ahead through this CTA's down tiles: waits (bounded) until the four epilogue warps of
     // every gate/up tile of the tile's 128 rows have published their H rows, then tells the
@@ -420,66 +436,84 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         acc_phase ^= 1u;
       }
     }
-  } else if (warp >= 2 && warp <= 5) {
+  } else if (warp >= kEpiWarp0) {
     // ------------------------------- epilogue --------------------------------------------------
-    // Results leave through a per-warp 4 KB staging buffer (32 rows x 128 bytes, 128-byte swizzle so
-    // the 16-byte writes of a warp hit distinct banks) and one TMA tensor store per buffer: the
-    // global writes are full lines and do not compete with the producers' loads for the SM's
-    // load/store path, which row-per-thread 16-byte stores did.
+    // Warps w and w + 4 read the same tensor-memory lane quadrant (rows quad*32 .. +31 of the tile)
+    // and split each row's columns.  The accumulator is copied raw into registers and released
+    // before any arithmetic, so the MMA issuer starts the next tile while this one is finished.
+    // Results leave through a per-quadrant 4 KB staging buffer (32 rows x 128 bytes, 128-byte
+    // swizzle so the 16-byte writes of a warp hit distinct banks; each warp of the pair fills its
+    // 64-byte half of every row) and one TMA tensor store per buffer: the global writes are full
+    // lines and do not compete with the producers' loads for the SM's load/store path.
     const int quad = warp & 3;                       // tensor-memory lanes this warp may read
+    const int half = (warp - kEpiWarp0) >> 2;        // which half of the columns
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-    const uint32_t stage_buf = smem_base + kStages * kStageBytes + (warp - 2) * kStoreBytes;
+    const uint32_t stage_buf = smem_base + kStages * kStageBytes + quad * kStoreBytes;
     const uint32_t my_line = stage_buf + lane * 128;
+    const bool issuer = half == 0 && lane == 0;      // the one thread of the pair that owns the TMA stores
+    const int pair_bar = 1 + quad;                   // named barrier of the pair (64 threads)
+    const int r_in_tile = quad * 32 + lane;
     uint32_t acc_phase = 0;
+    int par = 0;
     TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
     int side, x;
     while (it.next(side, x)) {
       const WorkItem w = decode_item(side, x, s_toff, G, p.side[side].NT);
-      const int row = w.row0 + quad * 32 + lane;
-      if (!mbar_wait(smem_u32(&s_acc_full), acc_phase, s_abort)) break;
+      const int row = w.row0 + r_in_tile;
+      // Both warps of a pair must take the same way out: they vote on the outcome of the wait.
+      const bool ok = mbar_wait(smem_u32(&s_acc_full), acc_phase, s_abort);
       acc_phase ^= 1u;
+      if (lane == 0) s_ok[par][quad][half] = ok ? 1 : 0;
+      pair_sync(pair_bar);
+      if (!(s_ok[par][quad][0] && s_ok[par][quad][1])) break;
       tc_fence_after();
       if (side == 0) {
-        float h[128];
+        // gate columns [64*half, +64) and the matching up columns of this thread's row
+        uint32_t g[2][32], u[2][32];
+        tmem_ld32(taddr + half * 64, g[0]);
+        tmem_ld32(taddr + half * 64 + 32, g[1]);
+        tmem_ld32(taddr + 128 + half * 64, u[0]);
+        tmem_ld32(taddr + 128 + half * 64 + 32, u[1]);
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));   // accumulator drained: the next tile may start
+        pin32(g[0]); pin32(g[1]); pin32(u[0]); pin32(u[1]);   // keep the arithmetic below the release
+        float h[64];
         float amax = 0.f;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t g[32], u[32];
-          tmem_ld32(taddr + c * 32, g);
-          tmem_ld32(taddr + 128 + c * 32, u);
-          tmem_wait_ld();
+        for (int c = 0; c < 2; ++c) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
-            const float gv = __uint_as_float(g[i]), uv = __uint_as_float(u[i]);
+            const float gv = __uint_as_float(g[c][i]), uv = __uint_as_float(u[c][i]);
             const float hv = __fdividef(gv, 1.f + __expf(-gv)) * uv;
             h[c * 32 + i] = hv;
             amax = fmaxf(amax, fabsf(hv));
           }
         }
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));   // accumulator drained: the next tile may start
+        s_amax[par][half][r_in_tile] = amax;
+        if (issuer) bulk_wait_read();                         // the previous store has left the buffer
+        pair_sync(pair_bar);
+        amax = fmaxf(amax, s_amax[par][half ^ 1][r_in_tile]);
         const int eps = pow2_scale_exponent(amax);
         const float inv = pow2_neg(eps);
-        if (lane == 0) bulk_wait_read();                      // the previous store has left the buffer
-        __syncwarp();
 #pragma unroll
-        for (int v = 0; v < 8; ++v) {
+        for (int v = 0; v < 4; ++v) {
           uint4 q;
           q.x = cvt_e4m3x4(h[16 * v + 0] * inv, h[16 * v + 1] * inv, h[16 * v + 2] * inv, h[16 * v + 3] * inv);
           q.y = cvt_e4m3x4(h[16 * v + 4] * inv, h[16 * v + 5] * inv, h[16 * v + 6] * inv, h[16 * v + 7] * inv);
           q.z = cvt_e4m3x4(h[16 * v + 8] * inv, h[16 * v + 9] * inv, h[16 * v + 10] * inv, h[16 * v + 11] * inv);
           q.w = cvt_e4m3x4(h[16 * v + 12] * inv, h[16 * v + 13] * inv, h[16 * v + 14] * inv, h[16 * v + 15] * inv);
-          st_shared_v4(my_line + ((v ^ (lane & 7)) << 4), q);
+          st_shared_v4(my_line + (((half * 4 + v) ^ (lane & 7)) << 4), q);
         }
-        p.h_sf[sf_index(row, w.nt, p.J_h)] = static_cast<uint8_t>(eps + 127);
+        if (half == 0) p.h_sf[sf_index(row, w.nt, p.J_h)] = static_cast<uint8_t>(eps + 127);
         fence_async_smem();
         if (fused) __threadfence();                            // the scale byte, before the counter below
-        __syncwarp();
-        if (lane == 0) {
+        pair_sync(pair_bar);
+        if (issuer) {
           tma_store_2d(&tmH, stage_buf, w.nt * 128, w.row0 + quad * 32);
           bulk_commit();
-          if (fused) {                                         // publish this warp's 32 rows of the H block
+          if (fused) {                                         // publish these 32 rows of the H block
             bulk_wait_all();
             asm volatile("fence.proxy.async;" ::: "memory");
             __threadfence();
@@ -487,43 +521,43 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
           }
         }
       } else {
-        // drain the accumulator into packed bf16 registers first, release it, then store
-        uint32_t packed[128];
+        // Of every 64-column group of the tile this thread takes 32 columns: [64*s + 32*half, +32).
+        uint32_t a[4][32];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          uint32_t a[32];
-          tmem_ld32(taddr + c * 32, a);
-          tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(a[2 * i]), __uint_as_float(a[2 * i + 1]));
-            packed[c * 16 + i] = *reinterpret_cast<const uint32_t*>(&b);
-          }
-        }
+        for (int s = 0; s < 4; ++s) tmem_ld32(taddr + s * 64 + half * 32, a[s]);
+        tmem_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));
+        pin32(a[0]); pin32(a[1]); pin32(a[2]); pin32(a[3]);
 #pragma unroll
-        for (int cg4 = 0; cg4 < 4; ++cg4) {                     // 64 columns = 128 bytes per row per store
-          if (w.nt * kBlockN + cg4 * 64 < p.d) {                // warp-uniform; the store clips at column d
-            if (lane == 0) bulk_wait_read();
-            __syncwarp();
+        for (int s = 0; s < 4; ++s) {                           // 64 columns = 128 bytes per row per store
+          if (w.nt * kBlockN + s * 64 < p.d) {                  // same for the pair; the store clips at column d
+            uint32_t packed[16];
 #pragma unroll
-            for (int v = 0; v < 8; ++v)
-              st_shared_v4(my_line + ((v ^ (lane & 7)) << 4),
-                           make_uint4(packed[cg4 * 32 + 4 * v], packed[cg4 * 32 + 4 * v + 1], packed[cg4 * 32 + 4 * v + 2],
-                                      packed[cg4 * 32 + 4 * v + 3]));
+            for (int i = 0; i < 16; ++i) {
+              const __nv_bfloat162 b =
+                  __floats2bfloat162_rn(__uint_as_float(a[s][2 * i]), __uint_as_float(a[s][2 * i + 1]));
+              packed[i] = *reinterpret_cast<const uint32_t*>(&b);
+            }
+            if (issuer) bulk_wait_read();
+            pair_sync(pair_bar);
+#pragma unroll
+            for (int v = 0; v < 4; ++v)
+              st_shared_v4(my_line + (((half * 4 + v) ^ (lane & 7)) << 4),
+                           make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]));
             fence_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-              tma_store_2d(&tmY, stage_buf, (w.nt * kBlockN + cg4 * 64) * 2, w.row0 + quad * 32);
+            pair_sync(pair_bar);
+            if (issuer) {
+              tma_store_2d(&tmY, stage_buf, (w.nt * kBlockN + s * 64) * 2, w.row0 + quad * 32);
               bulk_commit();
             }
           }
         }
       }
+      par ^= 1;
     }
-    if (lane == 0) bulk_wait_all();                             // stores still read the staging buffer
+    if (issuer) bulk_wait_all();                                // stores still read the staging buffer
     __syncwarp();
   }
 
