@@ -72,6 +72,13 @@ enum {
 };
 
 int tempo_version(void);
+
+/*
+ * [host] Which kernel steps 3a/3b/3 use from now on in this process: 0 = the default (one CTA per
+ * tile), 1 = one CTA per tile, 2 = CTA pairs.  For tests and measurements; results do not
+ * depend on it.  Not thread-safe against concurrent launches.  TEMPO_ERR_SHAPE for another value.
+ */
+int tempo_set_ffn_mode(int mode);
 const char* tempo_status_string(int code); /* [host] text for a TEMPO_ERR_* code */
 
 /* [host] Safe row capacity: round128(T*k) + 128*G_max (each instance pads by < 128 rows). */
@@ -171,6 +178,11 @@ int tempo_permute_pad(const tempo_shape* shape, const void* x_bf16, const int32_
  * stream never pauses between the two GEMMs.  The kernel's CTAs wait for each other's H blocks
  * (bounded, one per SM): launch it on a GPU it does not have to share with another long-running
  * kernel, or the wait may time out (TEMPO_STATUS_TIMEOUT).  Rows >= m_pad are not written.
+ * Two kernels implement step 3 with the same results: one CTA per 128x256 output tile (few rows per
+ * instance, the flat piece of Eq. 1) and pairs of CTAs on 256x256 tiles with the weight tile split
+ * between them (tcgen05 cta_group::2).  The first is the default for every shape: on B200 the pair
+ * kernel measured no faster with many rows and slower with few.  Either kernel is correct for any
+ * data and both give the same bits; see tempo_set_ffn_mode.
  */
 int tempo_ffn_gate_up(const tempo_shape* shape, const void* a_q, const uint8_t* a_sf, const void* packed,
                       const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf,

@@ -18,7 +18,7 @@ TEMPO_OK = 0
 STATUS_BAD_ID, STATUS_BAD_TABLE, STATUS_CAPACITY, STATUS_TIMEOUT, STATUS_BAD_SCALE = 1, 2, 4, 8, 16
 
 EXPORTS = (
-    "tempo_version", "tempo_status_string", "tempo_m_cap_bound", "tempo_sf_bytes", "tempo_workspace_bytes",
+    "tempo_version", "tempo_set_ffn_mode", "tempo_status_string", "tempo_m_cap_bound", "tempo_sf_bytes", "tempo_workspace_bytes",
     "tempo_packed_weight_bytes",
     "tempo_pack_weights", "tempo_count_dispatch", "tempo_count_dispatch_sampled", "tempo_permute_pad", "tempo_ffn_gate_up", "tempo_ffn_down",
     "tempo_grouped_ffn", "tempo_grouped_ffn_static", "tempo_unpermute_combine",
@@ -77,6 +77,10 @@ def make_shape(T, k, E, G_max, R_max, d, f, M_cap) -> TempoShape:
 
 def tempo_version() -> int:
     return _lib.tempo_version()
+
+
+def tempo_set_ffn_mode(mode: int) -> None:
+    _check(_lib.tempo_set_ffn_mode(ctypes.c_int(mode)), "tempo_set_ffn_mode")
 
 
 def tempo_m_cap_bound(shape: TempoShape) -> int:

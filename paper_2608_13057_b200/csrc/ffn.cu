@@ -32,222 +32,15 @@
 //
 // Every wait is bounded: after kWaitLimitNs the CTA raises an abort flag, all roles leave their
 // loops, TEMPO_STATUS_TIMEOUT is set and tensor memory is freed.
-#include <cuda.h>
-
-#include "tempo_kernels.cuh"
+#include "ffn_common.cuh"
 
 namespace tempo {
 
 constexpr int kStages = 4;
-constexpr int kBlockK = 128;
-constexpr int kBlockN = 256;
-constexpr int kABytes = kTileM * kBlockK;                 // 16 KB
-constexpr int kBBytes = kBlockN * kBlockK;                // 32 KB
-constexpr int kSfaBytes = 512;
-constexpr int kSfbBytes = 1024;
 constexpr int kStageBytes = kABytes + kBBytes + 2048;     // 51200, a multiple of 1024
 constexpr int kGemmThreads = 384;
 constexpr int kEpiWarp0 = 4;                               // first of the 8 epilogue warps
-constexpr int kTileOverhead = 5;                          // per-tile fixed cost in K-block steps (ramp + epilogue)
-constexpr int kTmemCols = 512;
-constexpr int kSfCol0 = 256;                              // scale slot s: A at 256+16s, B at 260+16s
-constexpr int kMaxSlots = 1024;
-constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
-constexpr int kStoreBytes = 32 * 128;                       // per-warp staging of a TMA store: 32 rows x 128 bytes
 constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 4 * kStoreBytes + 1024;
-
-
-// ---------------------------------------------------------------------------------------------
-// PTX wrappers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out of time).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  unsigned long long t0 = 0;
-  for (uint32_t it = 0;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 63u) {
-      if (*abort_flag) return false;
-      const unsigned long long now = global_timer_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
-    }
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1)
-      : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
-               : "memory");
-}
-// Same copy with an L2 evict-first hint: for weight tiles that are read once per launch.
-__device__ __forceinline__ void bulk_load_stream(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  uint64_t policy;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar), "l"(policy)
-      : "memory");
-}
-// TMA tensor store of a 32-row x 128-byte box from (swizzled) shared memory, bulk-group completion.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1)
-               : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_cp_sf(uint32_t tmem_addr, uint64_t desc) {
-  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(tmem_addr), "l"(desc) : "memory");
-}
-__device__ __forceinline__ void tc_mma_mxf8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Named barrier of two warps (64 threads).
-__device__ __forceinline__ void pair_sync(int id) { asm volatile("bar.sync %0, 64;" ::"r"(id) : "memory"); }
-// Compiler-level pin: the 32 values are treated as produced here, so nothing computed from them
-// can be scheduled above this point.
-__device__ __forceinline__ void pin32(uint32_t (&r)[32]) {
-#pragma unroll
-  for (int i = 0; i < 32; i += 8)
-    asm volatile("" : "+r"(r[i]), "+r"(r[i + 1]), "+r"(r[i + 2]), "+r"(r[i + 3]), "+r"(r[i + 4]), "+r"(r[i + 5]),
-                      "+r"(r[i + 6]), "+r"(r[i + 7])
-                 :: "memory");
-}
-
-// Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows of 128 bytes, groups of
-// 8 rows 1024 bytes apart (stride byte offset), descriptor version 1.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-  return static_cast<uint64_t>((addr >> 4) & 0x3fffu) | (1ull << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
-}
-// Descriptor of a 32-row x 16-byte scale atom (no swizzle, 8-row groups 128 bytes apart).
-__device__ __forceinline__ uint64_t smem_desc_sf(uint32_t addr) {
-  return static_cast<uint64_t>((addr >> 4) & 0x3fffu) | (static_cast<uint64_t>(128 >> 4) << 32) | (1ull << 46);
-}
-// Instruction descriptor of kind::mxf8f6f4.block_scale: A, B e4m3 (format 0), both K-major,
-// N >> 3 at bit 17, UE8M0 scales (bit 23), M >> 4 at bit 24; scale ids at bits 4 (B) and 29 (A).
-__device__ __forceinline__ uint32_t instr_desc(int sf_id) {
-  return (static_cast<uint32_t>(kBlockN >> 3) << 17) | (1u << 23) | (static_cast<uint32_t>(kTileM >> 4) << 24) |
-         (static_cast<uint32_t>(sf_id) << 29) | (static_cast<uint32_t>(sf_id) << 4);
-}
-
-struct WorkItem {
-  int side;      // 0 gate/up, 1 down
-  int inst, nt, row0, m_tiles;   // m_tiles: M-tiles of the instance (how often its B tiles are re-read)
-};
-
-// Tiles of one side are numbered instance-major, then N-tile, then M-tile, so CTAs running at the
-// same time share B tiles through L2 and an instance's A rows stay L2-resident across its N-tiles.
-__device__ __forceinline__ WorkItem decode_item(int side, int x, const int* toff, int G, int NT) {
-  int lo = 0, hi = G - 1;
-  while (lo < hi) {                       // first i with NT * toff[i+1] > x
-    const int mid = (lo + hi) >> 1;
-    if (NT * toff[mid + 1] > x) hi = mid; else lo = mid + 1;
-  }
-  const int local = x - NT * toff[lo];
-  const int Mi = toff[lo + 1] - toff[lo];
-  WorkItem w;
-  w.side = side;
-  w.inst = lo;
-  w.nt = local / Mi;
-  w.row0 = (toff[lo] + local % Mi) * kTileM;
-  w.m_tiles = Mi;
-  return w;
-}
-
-// Static tile assignment, the same arithmetic in every role of every CTA.
-//   gate/up tiles: x = c, c + C, ...  (n1 tiles; the first r1 = n1 % C CTAs get one more)
-//   down tiles:    dealt in rounds.  The CTAs WITHOUT the extra gate/up tile ("light") take part
-//                  in every round, the others only from round `lead` on, where `lead` is the extra
-//                  tile's cost in down tiles - so every CTA streams about the same bytes.
-struct TileIter {
-  int c, C, n1, n2, r1, light, lead;
-  int i1, round;
-  __device__ TileIter(int c_, int C_, int n1_, int n2_, int Kb1, int Kb2) {
-    c = c_; C = C_; n1 = n1_; n2 = n2_;
-    r1 = n1 % C;
-    light = C - r1;
-    lead = (r1 == 0 || n2 == 0) ? 0 : (2 * (Kb1 + kTileOverhead) + (Kb2 + kTileOverhead)) / (2 * (Kb2 + kTileOverhead));
-    i1 = c; round = 0;
-  }
-  // side and tile number of this CTA's next tile; false when it has none left
-  __device__ bool next(int& side, int& x) {
-    if (i1 < n1) { side = 0; x = i1; i1 += C; return true; }
-    for (;;) {
-      int y;
-      if (round < lead) {
-        if (c < r1) { round = lead; continue; }           // heavy CTAs skip the lead rounds
-        y = round * light + (c - r1);
-      } else {
-        y = lead * light + (round - lead) * C + c;
-      }
-      ++round;
-      if (y >= n2) return false;
-      side = 1; x = y;
-      return true;
-    }
-  }
-};
-
-__device__ __forceinline__ int ld_acquire(const int32_t* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
