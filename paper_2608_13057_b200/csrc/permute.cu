@@ -18,13 +18,12 @@ struct PermItem {
   uint4 lo, hi;
 };
 
-__device__ __forceinline__ void perm_load(const PermuteParams& p, long long gw, long long n_items, int chunks, int lane,
-                                          PermItem& it) {
-  it.live = gw < n_items;
-  it.row = it.live ? static_cast<int>(gw / chunks) : 0;
-  it.col = it.live ? static_cast<int>(gw % chunks) * 512 + lane * 16 : 0;
-  it.in = it.live && it.col < p.d;                  // d is a multiple of 128, so 8-lane groups agree
-  it.pair = it.live ? __ldg(p.row_pair + it.row) : -1;
+__device__ __forceinline__ void perm_load(const PermuteParams& p, int row, int chunk, bool live, int lane, PermItem& it) {
+  it.live = live;
+  it.row = live ? row : 0;
+  it.col = live ? chunk * 512 + lane * 16 : 0;
+  it.in = live && it.col < p.d;                     // d is a multiple of 128, so 8-lane groups agree
+  it.pair = live ? __ldg(p.row_pair + it.row) : -1;
   it.lo = make_uint4(0, 0, 0, 0);
   it.hi = make_uint4(0, 0, 0, 0);
 }
@@ -40,21 +39,24 @@ __device__ __forceinline__ void perm_gather(const PermuteParams& p, PermItem& it
 __device__ __forceinline__ void perm_finish(const PermuteParams& p, const PermItem& it, int lane, int J) {
   // padding rows come out as zero codes with scale 1 (all-zero block: eps = 0)
   const uint32_t w[8] = {it.lo.x, it.lo.y, it.lo.z, it.lo.w, it.hi.x, it.hi.y, it.hi.z, it.hi.w};
-  float v[16];
+  // block maximum on the packed bf16 pairs (magnitudes compare like the floats they stand for)
+  __nv_bfloat162 m2 = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[0]));
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-  }
-  float amax = 0.f;
-#pragma unroll
-  for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+  for (int i = 1; i < 8; ++i) m2 = __hmax2(m2, __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[i])));
+  const uint32_t mbits = *reinterpret_cast<const uint32_t*>(&m2);
+  float amax = fmaxf(__uint_as_float(mbits << 16), __uint_as_float(mbits & 0xffff0000u));
   amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
   amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
   amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
   if (!it.in) return;
   const int eps = pow2_scale_exponent(amax);
   const float inv = pow2_neg(eps);
+  float v[16];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
   uint4 q;
   q.x = cvt_e4m3x4(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv);
   q.y = cvt_e4m3x4(v[4] * inv, v[5] * inv, v[6] * inv, v[7] * inv);
@@ -71,16 +73,25 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_kernel(const Perm
   pdl_trigger();
   pdl_wait();
   const int m_pad = min(*p.m_pad, p.M_cap);
-  const long long n_items = static_cast<long long>(m_pad) * chunks;
-  const long long stride = static_cast<long long>(gridDim.x) * kPermWarps;
-  for (long long gw = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5); gw < n_items; gw += 2 * stride) {
+  // Item g = row * chunks + chunk; this warp takes g0, g0 + S, g0 + 2S, ... (S warps in the grid),
+  // two per trip.  Row and chunk of both are stepped by 2S with a carry instead of divided out.
+  const long long S = static_cast<long long>(gridDim.x) * kPermWarps;
+  const long long g0 = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5);
+  int row_a = static_cast<int>(g0 / chunks), ch_a = static_cast<int>(g0 % chunks);
+  int row_b = static_cast<int>((g0 + S) / chunks), ch_b = static_cast<int>((g0 + S) % chunks);
+  const int step_r = static_cast<int>((2 * S) / chunks), step_c = static_cast<int>((2 * S) % chunks);
+  while (row_a < m_pad) {
     PermItem a, b;
-    perm_load(p, gw, n_items, chunks, lane, a);
-    perm_load(p, gw + stride, n_items, chunks, lane, b);
+    perm_load(p, row_a, ch_a, true, lane, a);
+    perm_load(p, row_b, ch_b, row_b < m_pad, lane, b);
     perm_gather(p, a);
     perm_gather(p, b);
     perm_finish(p, a, lane, J);
     if (b.live) perm_finish(p, b, lane, J);
+    row_a += step_r; ch_a += step_c;
+    if (ch_a >= chunks) { ch_a -= chunks; ++row_a; }
+    row_b += step_r; ch_b += step_c;
+    if (ch_b >= chunks) { ch_b -= chunks; ++row_b; }
   }
 }
 
