@@ -28,7 +28,8 @@ Pins (tests/test_oracle_*.py): numpy.bincount and stable argsort for counts and 
 separately written sort-and-cut brute force for replica assignment, exact quota and
 bijection invariants, torch's CPU float8_e4m3fn cast for the code rounding, half-ulp error
 bounds and idempotence for the quantiser, torch fp32 dense SwiGLU MLP for the FFN, split
-invariance and linearity for the whole block.  No function here is "parity unpinned".
+invariance and linearity for the whole block; for the bf16 variant torch's CPU bfloat16 cast
+and the same dense-MLP and split-invariance checks.  No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -331,6 +332,57 @@ def expert_block(wl, M_cap=None, cum_counts=None):
         h_s = np.ones((M_cap, wl.f // QBLOCK), np.float32)
     out = combine(y, disp["pair_row"], wl.topk_w, wl.n_valid, wl.T, wl.k)
     return dict(disp, a_q=a_q, a_s=a_s, h_q=h_q, h_s=h_s, y=y, out=out)
+
+
+# ----------------------------------------------------------------------------------------
+# bf16 variant of steps 2-4 (the paper calibrates a bf16 grouped GEMM next to the fp8 one:
+# Section 2.1 and Table "Fitted cost parameters", row "DSv3 (bf16)")
+# ----------------------------------------------------------------------------------------
+# No quantiser: the gathered rows stay bf16, both GEMMs multiply bf16 values and accumulate wide,
+# and H is rounded to bf16 (round to nearest even) before the down GEMM, as a bf16 grouped-GEMM
+# pipeline stores it.  Pins: bf16_round against torch's CPU cast; the one-expert case against a
+# torch fp32 dense SwiGLU MLP; split invariance of the block.
+
+def bf16_round(v):
+    """f32 -> nearest bf16 (ties to even), returned as f32.  Finite inputs."""
+    b = np.ascontiguousarray(v, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    b = b + np.uint64(0x7FFF) + ((b >> np.uint64(16)) & np.uint64(1))
+    return ((b >> np.uint64(16)) << np.uint64(16)).astype(np.uint32).view(np.float32)
+
+
+def permute_pad_bf16(x, row_pair, m_pad, k):
+    """a f32 [M_cap, d] holding bf16 values: live rows are the token's row, every other row zero."""
+    x = np.asarray(x, dtype=np.float32)
+    a = np.zeros((len(row_pair), x.shape[1]), dtype=np.float32)
+    live = np.nonzero(np.asarray(row_pair[:int(m_pad)]) >= 0)[0]
+    if len(live):
+        a[live] = x[np.asarray(row_pair)[live] // k]
+    return a
+
+
+def expert_ffn_bf16(a, w13, w2):
+    """Rows of one expert instance, all inputs f32 arrays of bf16 values.  Returns (h bf16-valued f32, y f32)."""
+    f = w2.shape[1]
+    GU = (a.astype(np.float64) @ w13.astype(np.float64).T).astype(np.float32)
+    h = bf16_round(silu_f32(GU[:, :f]) * GU[:, f:])
+    y = (h.astype(np.float64) @ w2.astype(np.float64).T).astype(np.float32)
+    return h, y
+
+
+def expert_block_bf16(wl, M_cap=None):
+    """The block with the bf16 steps 2-4; dispatch and combine are those of expert_block."""
+    M_cap = wl.M_cap if M_cap is None else M_cap
+    disp = count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, M_cap)
+    a = permute_pad_bf16(wl.x, disp["row_pair"], disp["m_pad"], wl.k)
+    h = np.zeros((M_cap, wl.f), np.float32)
+    y = np.zeros((M_cap, wl.d), np.float32)
+    for i in range(wl.G_max):
+        lo, hi = int(disp["inst_off"][i]), int(disp["inst_off"][i + 1])
+        if hi > lo:
+            w13, w2 = wl.expert_weights_bf16(int(wl.slot_expert[i]))
+            h[lo:hi], y[lo:hi] = expert_ffn_bf16(a[lo:hi], w13, w2)
+    out = combine(y, disp["pair_row"], wl.topk_w, wl.n_valid, wl.T, wl.k)
+    return dict(disp, a=a, h=h, y=y, out=out)
 
 
 # ----------------------------------------------------------------------------------------

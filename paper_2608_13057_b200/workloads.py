@@ -75,6 +75,20 @@ class Workload:
     def drop_weight_cache(self) -> None:
         self._wcache.clear()
 
+    def expert_weights_bf16(self, e: int):
+        """(w13 f32 [2f, d], w2 f32 [d, f]) of the bf16 variant, not cached."""
+        return draw_expert_weights_bf16(self.weight_seed, e, self.d, self.f)
+
+    def slot_weights_bf16(self):
+        """Per-slot copies for the bf16 variant: (w13 f32 [G_max, 2f, d], w2 f32 [G_max, d, f])."""
+        w13 = np.zeros((self.G_max, 2 * self.f, self.d), np.float32)
+        w2 = np.zeros((self.G_max, self.d, self.f), np.float32)
+        for i in range(self.G_max):
+            e = int(self.slot_expert[i])
+            if e >= 0:
+                w13[i], w2[i] = self.expert_weights_bf16(e)
+        return w13, w2
+
     def slot_weights(self, slots: Optional[List[int]] = None):
         """Stack per-slot copies: every replica slot owns a copy of its expert's weights."""
         slots = list(range(self.G_max)) if slots is None else slots
@@ -120,6 +134,15 @@ def draw_expert_weights(weight_seed: int, e: int, d: int, f: int, std: float = 0
     w13_q, w13_s = _quantise_weight(w13)
     w2_q, w2_s = _quantise_weight(w2)
     return ExpertWeights(w13_q, w13_s, w2_q, w2_s)
+
+
+def draw_expert_weights_bf16(weight_seed: int, e: int, d: int, f: int, std: float = 0.02):
+    """The same draws as draw_expert_weights, rounded to bf16 instead (torch's CPU cast), as f32 arrays:
+    (w13 [2f, d], w2 [d, f]), every value exactly bf16-representable."""
+    g = _rng(weight_seed, _TAG_W, e)
+    w13 = torch.from_numpy(g.standard_normal((2 * f, d), dtype=np.float32)) * std
+    w2 = torch.from_numpy(g.standard_normal((d, f), dtype=np.float32)) * std
+    return (w13.to(torch.bfloat16).to(torch.float32).numpy(), w2.to(torch.bfloat16).to(torch.float32).numpy())
 
 
 def draw_activations(seed: int, T: int, d: int) -> np.ndarray:
