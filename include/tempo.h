@@ -224,6 +224,29 @@ int tempo_unpermute_combine(const tempo_shape* shape, const void* y_bf16, const 
                             const float* topk_w, const int32_t* n_valid, void* out_bf16, uint32_t* status,
                             void* stream);
 
+/*
+ * bf16 variant of steps 2 and 3 (the paper calibrates a bf16 grouped GEMM beside the fp8 one and finds
+ * the same two-regime shape with a later inflection: Section 2.1, Table "Fitted cost parameters").
+ * No quantiser: the gathered rows stay bf16, both GEMMs multiply bf16 values with fp32 accumulation
+ * on the tensor cores, H = silu(gate) * up is rounded to bf16 (nearest even) before the down GEMM,
+ * Y is stored as bf16.  Steps 1 and 4 are the calls above.
+ *   tempo_packed_weight_bytes_bf16 [host]  bytes of the packed bf16 blob (6*d*f per instance, padded)
+ *   tempo_pack_weights_bf16   one-time re-layout of w13 bf16 [G_max, 2f, d] (rows [0,f) gate, [f,2f) up)
+ *                             and w2 bf16 [G_max, d, f] into tiles of 256 rows x 64 values
+ *   tempo_permute_pad_bf16    a[row,:] = x[row_pair[row]/k, :], zero for rows without a pair; rows >= m_pad
+ *                             are not written.          out  a bf16 [M_cap, d]
+ *   tempo_grouped_ffn_bf16    both GEMMs in one kernel, as tempo_grouped_ffn (same `workspace`, same
+ *                             bounded waits and TEMPO_STATUS_TIMEOUT).   out  h bf16 [M_cap, f], y bf16 [M_cap, d]
+ */
+int tempo_packed_weight_bytes_bf16(const tempo_shape* shape /*[host]*/, size_t* bytes /*[host]*/);
+int tempo_pack_weights_bf16(const tempo_shape* shape, const void* w13_bf16, const void* w2_bf16, void* packed,
+                            void* stream);
+int tempo_permute_pad_bf16(const tempo_shape* shape, const void* x_bf16, const int32_t* row_pair,
+                           const int32_t* m_pad, void* a_bf16, uint32_t* status, void* stream);
+int tempo_grouped_ffn_bf16(const tempo_shape* shape, const void* a_bf16, const void* packed,
+                           const int32_t* inst_off, const int32_t* m_pad, void* h_bf16, void* y_bf16,
+                           uint32_t* status, void* workspace, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,6 +22,7 @@ EXPORTS = (
     "tempo_packed_weight_bytes",
     "tempo_pack_weights", "tempo_count_dispatch", "tempo_count_dispatch_sampled", "tempo_permute_pad", "tempo_ffn_gate_up", "tempo_ffn_down",
     "tempo_grouped_ffn", "tempo_grouped_ffn_static", "tempo_unpermute_combine",
+    "tempo_packed_weight_bytes_bf16", "tempo_pack_weights_bf16", "tempo_permute_pad_bf16", "tempo_grouped_ffn_bf16",
 )
 
 
@@ -180,6 +181,31 @@ def tempo_unpermute_combine(shape, y_bf16, pair_row, topk_w, n_valid, out_bf16, 
                                         _ptr(status, torch.int32), _stream()), "tempo_unpermute_combine")
 
 
+def tempo_packed_weight_bytes_bf16(shape: TempoShape) -> int:
+    out = ctypes.c_size_t(0)
+    _check(_lib.tempo_packed_weight_bytes_bf16(ctypes.byref(shape), ctypes.byref(out)), "tempo_packed_weight_bytes_bf16")
+    return out.value
+
+
+def tempo_pack_weights_bf16(shape, w13_bf16, w2_bf16, packed):
+    _check(_lib.tempo_pack_weights_bf16(ctypes.byref(shape), _ptr(w13_bf16, torch.bfloat16), _ptr(w2_bf16, torch.bfloat16),
+                                        _ptr(packed, torch.uint8), _stream()), "tempo_pack_weights_bf16")
+
+
+def tempo_permute_pad_bf16(shape, x_bf16, row_pair, m_pad, a_bf16, status):
+    _check(_lib.tempo_permute_pad_bf16(ctypes.byref(shape), _ptr(x_bf16, torch.bfloat16), _ptr(row_pair, torch.int32),
+                                       _ptr(m_pad, torch.int32), _ptr(a_bf16, torch.bfloat16), _ptr(status, torch.int32),
+                                       _stream()), "tempo_permute_pad_bf16")
+
+
+def tempo_grouped_ffn_bf16(shape, a_bf16, packed, inst_off, m_pad, h_bf16, y_bf16, status, workspace):
+    _check(_lib.tempo_grouped_ffn_bf16(ctypes.byref(shape), _ptr(a_bf16, torch.bfloat16), _ptr(packed, torch.uint8),
+                                       _ptr(inst_off, torch.int32), _ptr(m_pad, torch.int32),
+                                       _ptr(h_bf16, torch.bfloat16), _ptr(y_bf16, torch.bfloat16),
+                                       _ptr(status, torch.int32), _ptr(workspace, torch.uint8), _stream()),
+           "tempo_grouped_ffn_bf16")
+
+
 # ------------------------------------------------------------------------------------------------
 # A rank's device buffers: plain allocation and upload, no arithmetic.
 # ------------------------------------------------------------------------------------------------
@@ -238,6 +264,31 @@ class RankBuffers:
         tempo_permute_pad(s, self.x, self.row_pair, self.m_pad, self.a_q, self.a_sf, self.status)
         tempo_grouped_ffn(s, self.a_q, self.a_sf, packed, self.inst_off, self.m_pad, self.h_q, self.h_sf, self.y,
                           self.status, self.workspace)
+        tempo_unpermute_combine(s, self.y, self.pair_row, self.topk_w, self.n_valid, self.out, self.status)
+
+    # ---- bf16 variant (separate activation / weight buffers, allocated on first use) ----
+    def pack_weights_bf16(self, w13, w2):
+        dev = self.x.device
+        self.packed_bf16 = torch.empty(tempo_packed_weight_bytes_bf16(self.shape), dtype=torch.uint8, device=dev)
+        a = torch.as_tensor(w13).to(dev).to(torch.bfloat16).contiguous()
+        b = torch.as_tensor(w2).to(dev).to(torch.bfloat16).contiguous()
+        tempo_pack_weights_bf16(self.shape, a, b, self.packed_bf16)
+        torch.cuda.synchronize()
+        dev_kw = dict(dtype=torch.bfloat16, device=dev)
+        self.a_bf16 = torch.zeros(self.M_cap, self.d, **dev_kw)
+        self.h_bf16 = torch.zeros(self.M_cap, self.f, **dev_kw)
+        return self.packed_bf16
+
+    def run_block_bf16(self, packed=None):
+        """One pass of the block with the bf16 steps 2 and 3."""
+        s = self.shape
+        packed = self.packed_bf16 if packed is None else packed
+        tempo_count_dispatch(s, self.topk_ids, self.n_valid, self.replica_map, self.quota, self.cum_counts,
+                             self.counts, self.inst_count, self.inst_off, self.pair_row, self.row_pair,
+                             self.tile_inst, self.m_pad, self.status)
+        tempo_permute_pad_bf16(s, self.x, self.row_pair, self.m_pad, self.a_bf16, self.status)
+        tempo_grouped_ffn_bf16(s, self.a_bf16, packed, self.inst_off, self.m_pad, self.h_bf16, self.y, self.status,
+                               self.workspace)
         tempo_unpermute_combine(s, self.y, self.pair_row, self.topk_w, self.n_valid, self.out, self.status)
 
     def upload(self, wl, with_weights=True):

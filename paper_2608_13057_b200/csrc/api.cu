@@ -305,6 +305,68 @@ int tempo_grouped_ffn_static(const tempo_shape* s, const void* a_q, const uint8_
                          static_cast<cudaStream_t>(stream));
 }
 
+// ---- bf16 variant of steps 2 and 3 -------------------------------------------------------------------
+int tempo_packed_weight_bytes_bf16(const tempo_shape* s, size_t* bytes) {
+  if (bytes == nullptr) return TEMPO_ERR_NULL;
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  *bytes = pack_layout_bf16(s->G_max, s->d, s->f).total;
+  return TEMPO_OK;
+}
+
+int tempo_pack_weights_bf16(const tempo_shape* s, const void* w13_bf16, const void* w2_bf16, void* packed, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!w13_bf16 || !w2_bf16 || !packed) return TEMPO_ERR_NULL;
+  return launch_pack_bf16(s->G_max, s->d, s->f, static_cast<const __nv_bfloat16*>(w13_bf16),
+                          static_cast<const __nv_bfloat16*>(w2_bf16), static_cast<uint8_t*>(packed),
+                          static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+int tempo_permute_pad_bf16(const tempo_shape* s, const void* x_bf16, const int32_t* row_pair, const int32_t* m_pad,
+                           void* a_bf16, uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!x_bf16 || !row_pair || !m_pad || !a_bf16 || !status) return TEMPO_ERR_NULL;
+  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, m_pad, nullptr, nullptr};
+  return launch_permute_pad_bf16(p, static_cast<__nv_bfloat16*>(a_bf16), sm_count(), static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+int tempo_grouped_ffn_bf16(const tempo_shape* s, const void* a_bf16, const void* packed, const int32_t* inst_off,
+                           const int32_t* m_pad, void* h_bf16, void* y_bf16, uint32_t* status, void* workspace,
+                           void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!a_bf16 || !packed || !inst_off || !m_pad || !h_bf16 || !y_bf16 || !status || !workspace) return TEMPO_ERR_NULL;
+  const PackLayout L = pack_layout_bf16(s->G_max, s->d, s->f);
+  const uint8_t* blob = static_cast<const uint8_t*>(packed);
+  const int sms = sm_count();
+  if (sms <= 0) return TEMPO_ERR_CUDA;
+  CUtensorMap tmA1, tmA2, tmH, tmY;    // bf16 matrices seen as bytes: 2d / 2f per row
+  if (!make_map(&tmA1, a_bf16, s->M_cap, 2ull * s->d, 128)) return TEMPO_ERR_CUDA;
+  if (!make_map(&tmA2, h_bf16, s->M_cap, 2ull * s->f, 128)) return TEMPO_ERR_CUDA;
+  if (!make_map(&tmH, h_bf16, s->M_cap, 2ull * s->f, 32)) return TEMPO_ERR_CUDA;
+  if (!make_map(&tmY, y_bf16, s->M_cap, 2ull * s->d, 32)) return TEMPO_ERR_CUDA;
+  FfnParams p{};
+  p.side[0] = GemmSide{s->d / 64, 0, L.NT1, blob + L.off_w13, nullptr, nullptr};
+  p.side[1] = GemmSide{s->f / 64, 0, L.NT2, blob + L.off_w2, nullptr, nullptr};
+  p.run_mask = 3;
+  p.G_max = s->G_max;
+  p.M_cap = s->M_cap;
+  p.d = s->d;
+  p.f = s->f;
+  p.inst_off = inst_off;
+  p.m_pad = m_pad;
+  p.h_q = static_cast<uint8_t*>(h_bf16);
+  p.y = static_cast<__nv_bfloat16*>(y_bf16);
+  p.ready = static_cast<int32_t*>(workspace);
+  p.done = p.ready + s->M_cap / 128;
+  p.status = status;
+  return launch_ffn_bf16(tmA1, tmA2, tmH, tmY, p, sms, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK
+                                                                                                         : TEMPO_ERR_CUDA;
+}
+
 int tempo_unpermute_combine(const tempo_shape* s, const void* y_bf16, const int32_t* pair_row, const float* topk_w,
                             const int32_t* n_valid, void* out_bf16, uint32_t* status, void* stream) {
   const int rc = check_shape(s);

@@ -42,6 +42,10 @@ constexpr int kGemmThreads = 384;
 constexpr int kEpiWarp0 = 4;                               // first of the 8 epilogue warps
 constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 4 * kStoreBytes + 1024;
 
+// kBf16 = false: the fp8 path described above.  kBf16 = true: the bf16 variant (the paper calibrates a
+// bf16 grouped GEMM beside the fp8 one, Section 2.1): the same ring, roles and tiles with 64 bf16
+// values per 128-byte K-block, tcgen05.mma.kind::f16 without scales, and H stored as bf16.
+template <bool kBf16>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
            const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmY, const FfnParams p) {
@@ -112,7 +116,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
           if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
           const uint32_t full = smem_u32(&s_full[stage]);
           const uint32_t sB = smem_base + stage * kStageBytes + kABytes, sSF = sB + kBBytes;
-          const bool with_sf = (kb & 3) == 0;
+          const bool with_sf = !kBf16 && (kb & 3) == 0;
           mbar_arrive_expect_tx(full, kBBytes + (with_sf ? kSfbBytes : 0));
           if (stream_b) bulk_load_stream(sB, b_src + static_cast<size_t>(kb) * kBBytes, kBBytes, full);
           else bulk_load(sB, b_src + static_cast<size_t>(kb) * kBBytes, kBBytes, full);
@@ -154,7 +158,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
           if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
           const uint32_t full = smem_u32(&s_full[stage]);
           const uint32_t sA = smem_base + stage * kStageBytes, sSF = sA + kABytes + kBBytes;
-          const bool with_sf = (kb & 3) == 0;
+          const bool with_sf = !kBf16 && (kb & 3) == 0;
           mbar_arrive_expect_tx(full, kABytes + (with_sf ? kSfaBytes : 0));
           tma_load_2d(sA, tm, full, kb * kBlockK, w.row0);
           if (with_sf) bulk_load(sSF, sfa_src + static_cast<size_t>(kb >> 2) * kSfaBytes, kSfaBytes, full);
@@ -212,16 +216,22 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
           const uint32_t sA = smem_base + stage * kStageBytes, sB = sA + kABytes, sSF = sB + kBBytes;
           const uint32_t sfa_t = tmem_base + kSfCol0 + 16u * ((kb >> 2) & 1);
           const uint32_t sfb_t = sfa_t + 4;
-          if ((kb & 3) == 0) {
-            tc_cp_sf(sfa_t, smem_desc_sf(sSF));
-            tc_cp_sf(sfb_t, smem_desc_sf(sSF + kSfaBytes));
-            tc_cp_sf(sfb_t + 4, smem_desc_sf(sSF + kSfaBytes + 512));
-          }
-          const uint32_t idesc = instr_desc(kb & 3);
           const uint64_t da = smem_desc_sw128(sA), db = smem_desc_sw128(sB);
+          if constexpr (kBf16) {
 #pragma unroll
-          for (int ks = 0; ks < kBlockK / 32; ++ks)
-            tc_mma_mxf8(tmem_base, da + 2u * ks, db + 2u * ks, idesc, sfa_t, sfb_t, (kb | ks) != 0 ? 1u : 0u);
+            for (int ks = 0; ks < kBlockK / 32; ++ks)     // 16 bf16 values = 32 bytes per instruction
+              tc_mma_bf16(tmem_base, da + 2u * ks, db + 2u * ks, instr_desc_bf16(), (kb | ks) != 0 ? 1u : 0u);
+          } else {
+            if ((kb & 3) == 0) {
+              tc_cp_sf(sfa_t, smem_desc_sf(sSF));
+              tc_cp_sf(sfb_t, smem_desc_sf(sSF + kSfaBytes));
+              tc_cp_sf(sfb_t + 4, smem_desc_sf(sSF + kSfaBytes + 512));
+            }
+            const uint32_t idesc = instr_desc(kb & 3);
+#pragma unroll
+            for (int ks = 0; ks < kBlockK / 32; ++ks)
+              tc_mma_mxf8(tmem_base, da + 2u * ks, db + 2u * ks, idesc, sfa_t, sfb_t, (kb | ks) != 0 ? 1u : 0u);
+          }
           tc_commit(smem_u32(&s_empty[stage]));
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -260,7 +270,51 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       pair_sync(pair_bar);
       if (!(s_ok[par][quad][0] && s_ok[par][quad][1])) break;
       tc_fence_after();
-      if (side == 0) {
+      if (side == 0 && kBf16) {
+        // H columns [64*s + 32*half, +32), s = 0, 1: gate from the same accumulator columns, up 128
+        // columns further on; H leaves as bf16, 64 columns (128 bytes per row) per store.
+        uint32_t g[2][32], u[2][32];
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+          tmem_ld32(taddr + s * 64 + half * 32, g[s]);
+          tmem_ld32(taddr + 128 + s * 64 + half * 32, u[s]);
+        }
+        tmem_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));
+        pin32(g[0]); pin32(g[1]); pin32(u[0]); pin32(u[1]);
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+          uint32_t packed[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float g0 = __uint_as_float(g[s][2 * i]), g1 = __uint_as_float(g[s][2 * i + 1]);
+            const float h0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[s][2 * i]);
+            const float h1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[s][2 * i + 1]);
+            const __nv_bfloat162 b = __floats2bfloat162_rn(h0, h1);
+            packed[i] = *reinterpret_cast<const uint32_t*>(&b);
+          }
+          if (issuer) bulk_wait_read();
+          pair_sync(pair_bar);
+#pragma unroll
+          for (int v = 0; v < 4; ++v)
+            st_shared_v4(my_line + (((half * 4 + v) ^ (lane & 7)) << 4),
+                         make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]));
+          fence_async_smem();
+          pair_sync(pair_bar);
+          if (issuer) {
+            tma_store_2d(&tmH, stage_buf, (w.nt * 128 + s * 64) * 2, w.row0 + quad * 32);
+            bulk_commit();
+          }
+        }
+        if (issuer && fused) {                                 // publish these 32 rows of the H block
+          bulk_wait_all();
+          asm volatile("fence.proxy.async;" ::: "memory");
+          __threadfence();
+          atomicAdd(p.ready + (w.row0 >> 7), 1);
+        }
+      } else if (side == 0) {
         // gate columns [64*half, +64) and the matching up columns of this thread's row
         uint32_t g[2][32], u[2][32];
         tmem_ld32(taddr + half * 64, g[0]);
@@ -371,13 +425,24 @@ size_t ffn_workspace_bytes(int M_cap) {
   return ((2 * sizeof(int32_t) * static_cast<size_t>(M_cap / kTileM)) + 255) & ~static_cast<size_t>(255);
 }
 
-cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH, const CUtensorMap& tmY,
-                       const FfnParams& p, int num_sms, cudaStream_t stream) {
-  cudaError_t e = cudaFuncSetAttribute(ffn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+template <bool kBf16>
+static cudaError_t launch_ffn_t(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH,
+                                const CUtensorMap& tmY, const FfnParams& p, int num_sms, cudaStream_t stream) {
+  cudaError_t e = cudaFuncSetAttribute(ffn_kernel<kBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(kGemmSmemBytes));
   if (e != cudaSuccess) return e;
   const int grid = max(1, num_sms);   // one persistent CTA per SM; CTAs without work leave at once
-  return launch_pdl(ffn_kernel, dim3(grid), dim3(kGemmThreads), kGemmSmemBytes, stream, tmA1, tmA2, tmH, tmY, p);
+  return launch_pdl(ffn_kernel<kBf16>, dim3(grid), dim3(kGemmThreads), kGemmSmemBytes, stream, tmA1, tmA2, tmH, tmY, p);
+}
+
+cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH, const CUtensorMap& tmY,
+                       const FfnParams& p, int num_sms, cudaStream_t stream) {
+  return launch_ffn_t<false>(tmA1, tmA2, tmH, tmY, p, num_sms, stream);
+}
+
+cudaError_t launch_ffn_bf16(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH,
+                            const CUtensorMap& tmY, const FfnParams& p, int num_sms, cudaStream_t stream) {
+  return launch_ffn_t<true>(tmA1, tmA2, tmH, tmY, p, num_sms, stream);
 }
 
 }  // namespace tempo

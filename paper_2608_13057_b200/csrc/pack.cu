@@ -92,6 +92,52 @@ __global__ void pack_sf_kernel(const float* __restrict__ scales, uint8_t* __rest
   if (bad && threadIdx.x == 0) atomicOr(status, static_cast<uint32_t>(TEMPO_STATUS_BAD_SCALE));
 }
 
+// bf16 variant: W13 bf16 [G][2f][d] and W2 bf16 [G][d][f] into tiles of 256 rows x 64 values (128
+// bytes per row, 32 KB per tile), same row interleave, swizzle and tile order as the fp8 blob:
+//   W13t [G][f/128][d/64][256][128 B], then W2t [G][ceil(d/256)][f/64][256][128 B]; no scales.
+PackLayout pack_layout_bf16(int G, int d, int f) {
+  PackLayout L{};
+  L.NT1 = f / 128;
+  L.NT2 = (d + 255) / 256;
+  L.off_w13 = 0;
+  L.off_w2 = align1k(static_cast<size_t>(G) * 2 * f * d * 2);
+  L.total = align1k(L.off_w2 + static_cast<size_t>(G) * L.NT2 * 256 * f * 2);
+  L.off_sf13 = L.off_sf2 = L.total;
+  return L;
+}
+
+// One thread per 16-byte chunk (8 values).  Kb = K / 64.
+__global__ void pack_tiles_bf16_kernel(const __nv_bfloat16* __restrict__ src, uint8_t* __restrict__ dst, int G, int NT,
+                                       int Kb, int n_rows, int K, int mode) {
+  const size_t total = static_cast<size_t>(G) * NT * Kb * 256 * 8;
+  for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < total;
+       i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    const int c = static_cast<int>(i & 7);
+    const int r = static_cast<int>((i >> 3) & 255);
+    size_t rest = i >> 11;
+    const int kb = static_cast<int>(rest % Kb);
+    rest /= Kb;
+    const int nt = static_cast<int>(rest % NT);
+    const int g = static_cast<int>(rest / NT);
+    int srow;
+    if (mode == 0) srow = (r < 128 ? 0 : n_rows / 2) + nt * 128 + (r & 127);
+    else srow = nt * 256 + r;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (srow < n_rows)
+      v = *reinterpret_cast<const uint4*>(src + (static_cast<size_t>(g) * n_rows + srow) * K + kb * 64 + c * 8);
+    const size_t tile = (static_cast<size_t>(g) * NT + nt) * Kb + kb;
+    *reinterpret_cast<uint4*>(dst + tile * 32768 + r * 128 + ((c ^ (r & 7)) << 4)) = v;
+  }
+}
+
+cudaError_t launch_pack_bf16(int G, int d, int f, const __nv_bfloat16* w13, const __nv_bfloat16* w2, uint8_t* packed,
+                             cudaStream_t stream) {
+  const PackLayout L = pack_layout_bf16(G, d, f);
+  pack_tiles_bf16_kernel<<<2368, 256, 0, stream>>>(w13, packed + L.off_w13, G, L.NT1, d / 64, 2 * f, d, 0);
+  pack_tiles_bf16_kernel<<<2368, 256, 0, stream>>>(w2, packed + L.off_w2, G, L.NT2, f / 64, d, f, 1);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_pack(int G, int d, int f, const uint8_t* w13_q, const float* w13_s, const uint8_t* w2_q,
                         const float* w2_s, uint8_t* packed, uint32_t* status, cudaStream_t stream) {
   const PackLayout L = pack_layout(G, d, f);

@@ -95,6 +95,38 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_kernel(const Perm
   }
 }
 
+// bf16 variant of step 2: the gathered rows stay bf16 (no quantiser); rows without a pair are zero.
+// One warp per (row, 512-byte chunk), 16 bytes per lane.
+__global__ void __launch_bounds__(kPermWarps * 32) permute_pad_bf16_kernel(const PermuteParams p, __nv_bfloat16* a) {
+  const int lane = threadIdx.x & 31;
+  const int row_bytes = 2 * p.d;
+  const int chunks = (row_bytes + 511) >> 9;
+  pdl_trigger();
+  pdl_wait();
+  const int m_pad = min(*p.m_pad, p.M_cap);
+  const long long n_items = static_cast<long long>(m_pad) * chunks;
+  const long long stride = static_cast<long long>(gridDim.x) * kPermWarps;
+  for (long long gw = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5); gw < n_items; gw += stride) {
+    const int row = static_cast<int>(gw / chunks);
+    const int off = static_cast<int>(gw % chunks) * 512 + lane * 16;
+    if (off >= row_bytes) continue;
+    const int pair = __ldg(p.row_pair + row);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (pair >= 0)
+      v = __ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(p.x) +
+                                                static_cast<size_t>(pair / p.k) * row_bytes + off));
+    __stcs(reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(a) + static_cast<size_t>(row) * row_bytes + off), v);
+  }
+}
+
+cudaError_t launch_permute_pad_bf16(const PermuteParams& p, __nv_bfloat16* a, int num_sms, cudaStream_t stream) {
+  const long long warps = static_cast<long long>(p.M_cap) * ((2 * p.d + 511) >> 9);
+  long long blocks = (warps + kPermWarps - 1) / kPermWarps;
+  const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 8;
+  if (blocks > cap) blocks = cap;
+  return launch_pdl(permute_pad_bf16_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(kPermWarps * 32), 0, stream, p, a);
+}
+
 cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t stream) {
   const long long warps = static_cast<long long>(p.M_cap) * ((p.d + 511) >> 9);
   long long blocks = (warps + kPermWarps - 1) / kPermWarps;

@@ -56,6 +56,7 @@ struct PermuteParams {
   uint8_t* a_sf;
 };
 cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t stream);
+cudaError_t launch_permute_pad_bf16(const PermuteParams& p, __nv_bfloat16* a, int num_sms, cudaStream_t stream);
 
 struct CombineParams {
   int T, k, d;
@@ -72,6 +73,9 @@ struct PackLayout {
   int J1, J2, NT1, NT2;
 };
 PackLayout pack_layout(int G, int d, int f);
+PackLayout pack_layout_bf16(int G, int d, int f);   // off_w13, off_w2, NT1, NT2, total only
+cudaError_t launch_pack_bf16(int G, int d, int f, const __nv_bfloat16* w13, const __nv_bfloat16* w2, uint8_t* packed,
+                             cudaStream_t stream);
 cudaError_t launch_pack(int G, int d, int f, const uint8_t* w13_q, const float* w13_s, const uint8_t* w2_q,
                         const float* w2_s, uint8_t* packed, uint32_t* status, cudaStream_t stream);
 
@@ -101,6 +105,9 @@ struct FfnParams {
   uint32_t* status;
 };
 size_t ffn_workspace_bytes(int M_cap);
+// The bf16 variant: Kb counts 64-value K-blocks, the scale pointers and J_h are unused, h_q holds bf16.
+cudaError_t launch_ffn_bf16(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH,
+                            const CUtensorMap& tmY, const FfnParams& p, int num_sms, cudaStream_t stream);
 cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH, const CUtensorMap& tmY,
                        const FfnParams& p, int num_sms, cudaStream_t stream);
 
