@@ -190,19 +190,20 @@ def run_reference(args):
 # GPU arm
 # --------------------------------------------------------------------------------------------------
 
-def _capture_graphs(torch, buf, pools):
+def _capture_graphs(torch, buf, pools, run=None):
+    run = buf.run_block if run is None else run
     graphs = []
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
         for blob in pools:
-            buf.run_block(packed=blob)                  # warm the launch path outside capture
+            run(packed=blob)                            # warm the launch path outside capture
     torch.cuda.current_stream().wait_stream(side)
     torch.cuda.synchronize()
     for blob in pools:
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
-            buf.run_block(packed=blob)
+            run(packed=blob)
         graphs.append(g)
     return graphs
 
@@ -374,7 +375,8 @@ def run_sweep(args):
         # one weight set per G, copied into a rotation pool >> L2
         wl0 = W.config5_point(G, 1, with_x=False)
         probe = B.RankBuffers(G, 1, G, G, 1, d, f)
-        packed = probe.pack_weights(*wl0.slot_weights())
+        bf16 = args.variant == "bf16"
+        packed = probe.pack_weights_bf16(*wl0.slot_weights_bf16()) if bf16 else probe.pack_weights(*wl0.slot_weights())
         n_pools = min(64, max(2, math.ceil((1 << 30) / packed.numel())))
         pools = [packed] + [packed.clone() for _ in range(n_pools - 1)]
         del probe
@@ -386,14 +388,20 @@ def run_sweep(args):
             buf.replica_map.copy_(torch.arange(G, device="cuda", dtype=torch.int32).view(G, 1))
             buf.quota.fill_(N)
             buf.x.copy_(torch.randn(T, d, generator=gen, device="cuda").to(torch.bfloat16))
-            graphs = _capture_graphs(torch, buf, pools)
+            if bf16:
+                buf.alloc_bf16()
+            graphs = _capture_graphs(torch, buf, pools, buf.run_block_bf16 if bf16 else None)
             s = buf.shape
             ffn_graphs = []
             for blob in pools:
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g):
-                    B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
-                                        buf.status, buf.workspace)
+                    if bf16:
+                        B.tempo_grouped_ffn_bf16(s, buf.a_bf16, blob, buf.inst_off, buf.m_pad, buf.h_bf16, buf.y,
+                                                 buf.status, buf.workspace)
+                    else:
+                        B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf,
+                                            buf.y, buf.status, buf.workspace)
                 ffn_graphs.append(g)
 
             def med(gs):
@@ -422,7 +430,7 @@ def run_sweep(args):
     G = np.array([r["G"] for r in rows])
     N = np.array([r["N"] for r in rows])
     tiles = np.array([r["tiles"] for r in rows])
-    result = {"sweep": {"d": d, "f": f, "points": len(rows), "replays": replays}, "rows": rows}
+    result = {"sweep": {"d": d, "f": f, "points": len(rows), "replays": replays, "variant": args.variant}, "rows": rows}
     for scope in ("ffn", "block"):
         t = np.array([r[f"t_{scope}_us"] for r in rows])
         result[f"fit_{scope}"] = C.fit_max_affine(G, N, t)
@@ -442,6 +450,7 @@ def main():
     ap.add_argument("--sweep-G", default="")
     ap.add_argument("--sweep-N", default="")
     ap.add_argument("--replays", type=int, default=30)
+    ap.add_argument("--variant", default="fp8", choices=["fp8", "bf16"], help="--sweep only: which steps 2 and 3")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

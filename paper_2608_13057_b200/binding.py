@@ -274,10 +274,13 @@ class RankBuffers:
         b = torch.as_tensor(w2).to(dev).to(torch.bfloat16).contiguous()
         tempo_pack_weights_bf16(self.shape, a, b, self.packed_bf16)
         torch.cuda.synchronize()
-        dev_kw = dict(dtype=torch.bfloat16, device=dev)
+        self.alloc_bf16()
+        return self.packed_bf16
+
+    def alloc_bf16(self):
+        dev_kw = dict(dtype=torch.bfloat16, device=self.x.device)
         self.a_bf16 = torch.zeros(self.M_cap, self.d, **dev_kw)
         self.h_bf16 = torch.zeros(self.M_cap, self.f, **dev_kw)
-        return self.packed_bf16
 
     def run_block_bf16(self, packed=None):
         """One pass of the block with the bf16 steps 2 and 3."""
