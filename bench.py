@@ -58,6 +58,9 @@ def make_workload(name: str, rank: int = 0):
         return W.config3(name[5:].replace("-", "_"), seed=2 + 101 * rank)
     if name == "cfg4":
         return W.config4(seed=3 + 101 * rank)
+    if name.startswith("cfg5s-"):                      # cfg5s-G-N: same totals, uneven rows per instance
+        _, G, N = name.split("-")
+        return W.config5_skewed(int(G), int(N))
     if name.startswith("cfg5-"):                       # cfg5-G-N
         _, G, N = name.split("-")
         return W.config5_point(int(G), int(N))

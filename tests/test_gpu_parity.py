@@ -309,6 +309,15 @@ def test_sweep_points_sampled(B, G, N):
     _sampled_rows_check(B, wl, buf, rows_per_inst=2, n_tokens=8)
 
 
+def test_skewed_sweep_point_sampled(B):
+    """Same totals as a sweep point, rows spread unevenly over the instances (227 ... 1824 rows)."""
+    wl = W.config5_skewed(8, 1024)
+    buf = _run_block(B, wl)
+    ref = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    _sampled_rows_check(B, wl, buf, rows_per_inst=2, n_tokens=8)
+
+
 def test_block_is_reproducible_run_to_run(B):
     wl = W.config2()
     buf = _run_block(B, wl)
