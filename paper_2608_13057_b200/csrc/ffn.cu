@@ -151,8 +151,11 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
             }
           }
           if (!ok) break;
-          __threadfence();
-          asm volatile("fence.proxy.async;" ::: "memory");   // H was written by ordinary stores, TMA reads it
+          // The scout's acquire load saw the rows published; its word reaches this thread through
+          // shared memory (block-scope fences on both sides), then the proxy fence orders the
+          // ordinary stores that wrote H before the TMA reads below.
+          __threadfence_block();
+          asm volatile("fence.proxy.async;" ::: "memory");
         }
         for (int kb = 0; kb < gs.Kb; ++kb) {
           if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
@@ -191,12 +194,12 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
           }
         }
         if (!ok) break;
+        __threadfence_block();
+        *s_dep = ++cleared;                      // tell the producer first, then do the bookkeeping
         if (atomicAdd(p.done + tau, 1) == p.side[1].NT - 1) {
           atomicExch(p.ready + tau, 0);
           atomicExch(p.done + tau, 0);
         }
-        __threadfence();
-        *s_dep = ++cleared;
       }
     }
   } else if (warp == 1) {
@@ -284,16 +287,26 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));
         pin32(g[0]); pin32(g[1]); pin32(u[0]); pin32(u[1]);
+        uint32_t any_gate = 0;                               // all-zero gate row (padding): H = 0, skip the exponentials
+#pragma unroll
+        for (int s = 0; s < 2; ++s)
+#pragma unroll
+          for (int i = 0; i < 32; ++i) any_gate |= g[s][i];
+        const bool live_row = (any_gate & 0x7fffffffu) != 0;
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
           uint32_t packed[16];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float g0 = __uint_as_float(g[s][2 * i]), g1 = __uint_as_float(g[s][2 * i + 1]);
-            const float h0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[s][2 * i]);
-            const float h1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[s][2 * i + 1]);
-            const __nv_bfloat162 b = __floats2bfloat162_rn(h0, h1);
-            packed[i] = *reinterpret_cast<const uint32_t*>(&b);
+          for (int i = 0; i < 16; ++i) packed[i] = 0;
+          if (live_row) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float g0 = __uint_as_float(g[s][2 * i]), g1 = __uint_as_float(g[s][2 * i + 1]);
+              const float h0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(u[s][2 * i]);
+              const float h1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(u[s][2 * i + 1]);
+              const __nv_bfloat162 b = __floats2bfloat162_rn(h0, h1);
+              packed[i] = *reinterpret_cast<const uint32_t*>(&b);
+            }
           }
           if (issuer) bulk_wait_read();
           pair_sync(pair_bar);
@@ -326,43 +339,52 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&s_acc_empty));   // accumulator drained: the next tile may start
         pin32(g[0]); pin32(g[1]); pin32(u[0]); pin32(u[1]);   // keep the arithmetic below the release
-        float h[64];
         float amax = 0.f;
+        // A row whose gate values are all zero (a padding row: its activations are zero) gives
+        // H = 0 whatever `up` holds; with few live rows per tile most rows are like that, and
+        // skipping their exponentials shortens the wait of the down tiles that need this H block.
+        // H overwrites the gate registers (an all-zero gate row already is its own H).
+        uint32_t any_gate = 0;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float gv = __uint_as_float(g[c][i]), uv = __uint_as_float(u[c][i]);
-            const float hv = __fdividef(gv, 1.f + __expf(-gv)) * uv;
-            h[c * 32 + i] = hv;
-            amax = fmaxf(amax, fabsf(hv));
+          for (int i = 0; i < 32; ++i) any_gate |= g[c][i];
+        if ((any_gate & 0x7fffffffu) != 0) {
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float gv = __uint_as_float(g[c][i]), uv = __uint_as_float(u[c][i]);
+              const float hv = __fdividef(gv, 1.f + __expf(-gv)) * uv;
+              g[c][i] = __float_as_uint(hv);
+              amax = fmaxf(amax, fabsf(hv));
+            }
           }
         }
+#define TEMPO_H(j) __uint_as_float(g[(j) >> 5][(j) & 31])
         s_amax[par][half][r_in_tile] = amax;
-        if (issuer) bulk_wait_read();                         // the previous store has left the buffer
         pair_sync(pair_bar);
         amax = fmaxf(amax, s_amax[par][half ^ 1][r_in_tile]);
         const int eps = pow2_scale_exponent(amax);
         const float inv = pow2_neg(eps);
+        // H goes out with ordinary 16-byte stores (64 bytes of the row per thread), not through the
+        // TMA unit: there a store queues behind the weight loads already issued for the next tile,
+        // which held the H block back by 4-9 us while down tiles of other CTAs waited for it.
+        uint4* dst = reinterpret_cast<uint4*>(p.h_q + static_cast<size_t>(row) * p.f + w.nt * 128 + half * 64);
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           uint4 q;
-          q.x = cvt_e4m3x4(h[16 * v + 0] * inv, h[16 * v + 1] * inv, h[16 * v + 2] * inv, h[16 * v + 3] * inv);
-          q.y = cvt_e4m3x4(h[16 * v + 4] * inv, h[16 * v + 5] * inv, h[16 * v + 6] * inv, h[16 * v + 7] * inv);
-          q.z = cvt_e4m3x4(h[16 * v + 8] * inv, h[16 * v + 9] * inv, h[16 * v + 10] * inv, h[16 * v + 11] * inv);
-          q.w = cvt_e4m3x4(h[16 * v + 12] * inv, h[16 * v + 13] * inv, h[16 * v + 14] * inv, h[16 * v + 15] * inv);
-          st_shared_v4(my_line + (((half * 4 + v) ^ (lane & 7)) << 4), q);
+          q.x = cvt_e4m3x4(TEMPO_H(16 * v + 0) * inv, TEMPO_H(16 * v + 1) * inv, TEMPO_H(16 * v + 2) * inv, TEMPO_H(16 * v + 3) * inv);
+          q.y = cvt_e4m3x4(TEMPO_H(16 * v + 4) * inv, TEMPO_H(16 * v + 5) * inv, TEMPO_H(16 * v + 6) * inv, TEMPO_H(16 * v + 7) * inv);
+          q.z = cvt_e4m3x4(TEMPO_H(16 * v + 8) * inv, TEMPO_H(16 * v + 9) * inv, TEMPO_H(16 * v + 10) * inv, TEMPO_H(16 * v + 11) * inv);
+          q.w = cvt_e4m3x4(TEMPO_H(16 * v + 12) * inv, TEMPO_H(16 * v + 13) * inv, TEMPO_H(16 * v + 14) * inv, TEMPO_H(16 * v + 15) * inv);
+          dst[v] = q;
         }
+#undef TEMPO_H
         if (half == 0) p.h_sf[sf_index(row, w.nt, p.J_h)] = static_cast<uint8_t>(eps + 127);
-        fence_async_smem();
-        if (fused) __threadfence();                            // the scale byte, before the counter below
-        pair_sync(pair_bar);
-        if (issuer) {
-          tma_store_2d(&tmH, stage_buf, w.nt * 128, w.row0 + quad * 32);
-          bulk_commit();
-          if (fused) {                                         // publish these 32 rows of the H block
-            bulk_wait_all();
-            asm volatile("fence.proxy.async;" ::: "memory");
+        if (fused) {                                           // publish these 32 rows of the H block:
+          pair_sync(pair_bar);                                 // both warps' stores are issued, then one
+          if (issuer) {                                        // thread fences for the pair and bumps the counter
             __threadfence();
             atomicAdd(p.ready + (w.row0 >> 7), 1);
           }

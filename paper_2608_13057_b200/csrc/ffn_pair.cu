@@ -416,18 +416,29 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant_
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(acc_empty_leader);
         pin32(g[0]); pin32(g[1]); pin32(u[0]); pin32(u[1]);
-        float h[64];
         float amax = 0.f;
+        // A row whose gate values are all zero (a padding row: its activations are zero) gives
+        // H = 0 whatever `up` holds; with few live rows per tile most rows are like that, and
+        // skipping their exponentials shortens the wait of the down tiles that need this H block.
+        // H overwrites the gate registers (an all-zero gate row already is its own H).
+        uint32_t any_gate = 0;
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float gv = __uint_as_float(g[c][i]), uv = __uint_as_float(u[c][i]);
-            const float hv = __fdividef(gv, 1.f + __expf(-gv)) * uv;
-            h[c * 32 + i] = hv;
-            amax = fmaxf(amax, fabsf(hv));
+          for (int i = 0; i < 32; ++i) any_gate |= g[c][i];
+        if ((any_gate & 0x7fffffffu) != 0) {
+#pragma unroll
+          for (int c = 0; c < 2; ++c) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float gv = __uint_as_float(g[c][i]), uv = __uint_as_float(u[c][i]);
+              const float hv = __fdividef(gv, 1.f + __expf(-gv)) * uv;
+              g[c][i] = __float_as_uint(hv);
+              amax = fmaxf(amax, fabsf(hv));
+            }
           }
         }
+#define TEMPO_H(j) __uint_as_float(g[(j) >> 5][(j) & 31])
         s_amax[par][half][r_in_tile] = amax;
         if (issuer) bulk_wait_read();
         pair_sync(pair_bar);
@@ -437,12 +448,13 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant_
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           uint4 q;
-          q.x = cvt_e4m3x4(h[16 * v + 0] * inv, h[16 * v + 1] * inv, h[16 * v + 2] * inv, h[16 * v + 3] * inv);
-          q.y = cvt_e4m3x4(h[16 * v + 4] * inv, h[16 * v + 5] * inv, h[16 * v + 6] * inv, h[16 * v + 7] * inv);
-          q.z = cvt_e4m3x4(h[16 * v + 8] * inv, h[16 * v + 9] * inv, h[16 * v + 10] * inv, h[16 * v + 11] * inv);
-          q.w = cvt_e4m3x4(h[16 * v + 12] * inv, h[16 * v + 13] * inv, h[16 * v + 14] * inv, h[16 * v + 15] * inv);
+          q.x = cvt_e4m3x4(TEMPO_H(16 * v + 0) * inv, TEMPO_H(16 * v + 1) * inv, TEMPO_H(16 * v + 2) * inv, TEMPO_H(16 * v + 3) * inv);
+          q.y = cvt_e4m3x4(TEMPO_H(16 * v + 4) * inv, TEMPO_H(16 * v + 5) * inv, TEMPO_H(16 * v + 6) * inv, TEMPO_H(16 * v + 7) * inv);
+          q.z = cvt_e4m3x4(TEMPO_H(16 * v + 8) * inv, TEMPO_H(16 * v + 9) * inv, TEMPO_H(16 * v + 10) * inv, TEMPO_H(16 * v + 11) * inv);
+          q.w = cvt_e4m3x4(TEMPO_H(16 * v + 12) * inv, TEMPO_H(16 * v + 13) * inv, TEMPO_H(16 * v + 14) * inv, TEMPO_H(16 * v + 15) * inv);
           st_shared_v4(my_line + (((half * 4 + v) ^ (lane & 7)) << 4), q);
         }
+#undef TEMPO_H
         if (half == 0) p.h_sf[sf_index(row, w.nt, p.J_h)] = static_cast<uint8_t>(eps + 127);
         fence_async_smem();
         if (fused) __threadfence();
