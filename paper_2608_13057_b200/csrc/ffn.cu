@@ -26,7 +26,10 @@
 //   warps 4-11 epilogue, two warps per tensor-memory lane quadrant, each taking half of a row's
 //              columns: tcgen05.ld the raw accumulator into registers and hand tensor memory back
 //              to the MMA issuer at once, then the math (the pair shares the row maximum through
-//              shared memory), swizzled staging in shared memory, TMA tensor stores
+//              shared memory).  Y leaves through swizzled staging in shared memory and TMA tensor
+//              stores; H leaves through ordinary 16-byte stores, because other CTAs wait for it and
+//              a TMA store queues behind the weight loads already issued for the next tile (tmH is
+//              not used by this kernel; the CTA-pair kernel takes the same four maps and uses it)
 // Scales are UE8M0 per 128 K-elements; the MMA takes one scale byte per row (A) and per column
 // (B) for each K=32 step, so the four steps of a K-block select the same byte (scale id kb % 4).
 //
@@ -77,7 +80,6 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA1)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA2)) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmH)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
   }
   if (warp == 1) {
@@ -275,7 +277,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       tc_fence_after();
       if (side == 0 && kBf16) {
         // H columns [64*s + 32*half, +32), s = 0, 1: gate from the same accumulator columns, up 128
-        // columns further on; H leaves as bf16, 64 columns (128 bytes per row) per store.
+        // columns further on; H leaves as bf16, 64 bytes of the row per thread and step.
         uint32_t g[2][32], u[2][32];
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
@@ -308,24 +310,17 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
               packed[i] = *reinterpret_cast<const uint32_t*>(&b);
             }
           }
-          if (issuer) bulk_wait_read();
-          pair_sync(pair_bar);
+          // ordinary stores, as for the fp8 H (a TMA store would queue behind the next tile's weight loads)
+          uint4* dst = reinterpret_cast<uint4*>(p.h_q + (static_cast<size_t>(row) * p.f + w.nt * 128 + s * 64 + half * 32) * 2);
 #pragma unroll
-          for (int v = 0; v < 4; ++v)
-            st_shared_v4(my_line + (((half * 4 + v) ^ (lane & 7)) << 4),
-                         make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]));
-          fence_async_smem();
+          for (int v = 0; v < 4; ++v) dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+        }
+        if (fused) {                                           // publish these 32 rows of the H block
           pair_sync(pair_bar);
           if (issuer) {
-            tma_store_2d(&tmH, stage_buf, (w.nt * 128 + s * 64) * 2, w.row0 + quad * 32);
-            bulk_commit();
+            __threadfence();
+            atomicAdd(p.ready + (w.row0 >> 7), 1);
           }
-        }
-        if (issuer && fused) {                                 // publish these 32 rows of the H block
-          bulk_wait_all();
-          asm volatile("fence.proxy.async;" ::: "memory");
-          __threadfence();
-          atomicAdd(p.ready + (w.row0 >> 7), 1);
         }
       } else if (side == 0) {
         // gate columns [64*half, +64) and the matching up columns of this thread's row
