@@ -61,6 +61,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   __shared__ int s_abort_storage;
   __shared__ int s_dep_storage;
   __shared__ int s_toff[kMaxSlots + 1];
+  __shared__ uint16_t s_cold[kMaxSlots + 2];   // M-tiles of cold instances before each instance (at most 2 each)
   __shared__ float s_amax[2][2][kTileM];   // [tile parity][column half][row]: row maxima of the two half-row warps
   __shared__ int s_ok[2][4][2];             // [tile parity][quadrant][column half]: that warp's wait succeeded
   volatile int* s_abort = &s_abort_storage;
@@ -96,10 +97,29 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   const int Kb1 = p.side[0].Kb, Kb2 = p.side[1].Kb;
 
   for (int i = tid; i <= G; i += kGemmThreads) s_toff[i] = max(0, min(p.inst_off[i], m_pad)) >> 7;
+  __syncthreads();
+  if (warp == 0) {   // cold[i] = M-tiles of cold instances before instance i
+    int carry = 0;
+    for (int base = 0; base < G; base += 32) {
+      const int i = base + lane;
+      const int Mi = i < G ? s_toff[i + 1] - s_toff[i] : 0;
+      const int c = Mi <= kColdTiles ? Mi : 0;
+      int incl = c;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (i < G) s_cold[i] = static_cast<uint16_t>(carry + incl - c);
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) s_cold[G] = static_cast<uint16_t>(carry);
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
+  const int cold_tiles = s_cold[G], hot_tiles = m_tiles - cold_tiles;
+  const TileOrder order1(p.side[0].NT, hot_tiles, cold_tiles, gridDim.x), order2(p.side[1].NT, hot_tiles, cold_tiles, gridDim.x);
 
   if (warp == 0) {
     // ------------------------------- weight producer ------------------------------------------
@@ -110,7 +130,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       int side, x;
       while (ok && it.next(side, x)) {
         const GemmSide& gs = p.side[side];
-        const WorkItem w = decode_item(side, x, s_toff, G, gs.NT);
+        const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2);
         const uint8_t* sfb_src = gs.sfb + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.JK * kSfbBytes;
         const uint8_t* b_src = gs.wt + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.Kb * kBBytes;
         const bool stream_b = w.m_tiles <= 2;
@@ -137,7 +157,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       int side, x;
       while (ok && it.next(side, x)) {
         const GemmSide& gs = p.side[side];
-        const WorkItem w = decode_item(side, x, s_toff, G, gs.NT);
+        const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2);
         const uint8_t* sfa_src = gs.sfa + static_cast<size_t>(w.row0 >> 7) * gs.JK * kSfaBytes;
         const CUtensorMap* tm = side == 0 ? &tmA1 : &tmA2;
         if (side == 1 && fused) {
@@ -184,7 +204,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       bool ok = true;
       while (ok && it.next(side, x)) {
         if (side == 0) continue;
-        const WorkItem w = decode_item(1, x, s_toff, G, p.side[1].NT);
+        const WorkItem w = decode_item(1, x, s_toff, s_cold, G, order2);
         const int tau = w.row0 >> 7;
         unsigned long long t0 = 0;
         for (uint32_t spin = 0; ld_acquire(p.ready + tau) < want; ++spin) {
@@ -266,7 +286,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
     int side, x;
     while (it.next(side, x)) {
-      const WorkItem w = decode_item(side, x, s_toff, G, p.side[side].NT);
+      const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2);
       const int row = w.row0 + r_in_tile;
       // Both warps of a pair must take the same way out: they vote on the outcome of the wait.
       const bool ok = mbar_wait(smem_u32(&s_acc_full), acc_phase, s_abort);

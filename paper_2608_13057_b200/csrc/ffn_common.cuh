@@ -175,13 +175,58 @@ struct WorkItem {
 
 // Tiles of one side are numbered instance-major, then N-tile, then M-tile, so CTAs running at the
 // same time share B tiles through L2 and an instance's A rows stay L2-resident across its N-tiles.
-__device__ __forceinline__ WorkItem decode_item(int side, int x, const int* toff, int G, int NT) {
-  int lo = 0, hi = G - 1;
-  while (lo < hi) {                       // first i with NT * toff[i+1] > x
-    const int mid = (lo + hi) >> 1;
-    if (NT * toff[mid + 1] > x) hi = mid; else lo = mid + 1;
+//
+// Two classes of instances are numbered separately: COLD ones (at most kColdTiles M-tiles: their
+// weights are read from HBM and hardly re-used) and HOT ones (their weights are re-read from L2 by
+// many M-tiles, so a tile is bound by the operand bytes an SM takes in).  A batch that has both
+// (the hot/cold mix an EPLB-style placement leaves on a rank) would otherwise run its hot tiles
+// with HBM idle and then its cold tiles with the tensor pipes idle.  TileOrder deals every wave of
+// C tiles partly from the hot list and partly from the cold list, in the ratio at which a cold
+// tile's weight stream and a hot tile's operand intake take the same time, so both run at once.
+// With only one class present the order is the plain numbering.
+constexpr int kColdTiles = 2;
+constexpr int kColdShareNum = 80, kColdShareDen = 148;   // CTAs on cold tiles: HBM rate x hot-tile time / tile bytes
+
+struct TileOrder {          // of one side
+  int NT, n_hot, n_cold, C, Ch, Cc, W;
+  __device__ TileOrder(int NT_, int hot_tiles, int cold_tiles, int C_) {
+    NT = NT_; C = C_;
+    n_hot = hot_tiles * NT; n_cold = cold_tiles * NT;
+    Cc = (n_hot == 0 || n_cold == 0) ? 0 : max(1, min(C - 1, (C * kColdShareNum) / kColdShareDen));
+    Ch = C - Cc;
+    W = Cc == 0 ? 0 : min(n_hot / Ch, n_cold / Cc);      // waves dealt from both lists
   }
-  const int local = x - NT * toff[lo];
+  // v-th tile of the side -> (class, index in the class's list)
+  __device__ void map(int v, bool& cold, int& k) const {
+    if (n_cold == 0) { cold = false; k = v; return; }
+    if (n_hot == 0) { cold = true; k = v; return; }
+    if (v < W * C) {
+      const int w = v / C, j = v - w * C;
+      if (j < Ch) { cold = false; k = w * Ch + j; } else { cold = true; k = w * Cc + (j - Ch); }
+      return;
+    }
+    const int r = v - W * C, rem_hot = n_hot - W * Ch;     // what is left: hot first, then cold
+    if (r < rem_hot) { cold = false; k = W * Ch + r; } else { cold = true; k = W * Cc + (r - rem_hot); }
+  }
+};
+
+// M-tiles of the class before instance i: cold_before[i] counts the tiles of cold instances.
+__device__ __forceinline__ int class_before(const int* toff, const uint16_t* cold_before, bool cold, int i) {
+  return cold ? static_cast<int>(cold_before[i]) : toff[i] - static_cast<int>(cold_before[i]);
+}
+
+__device__ __forceinline__ WorkItem decode_item(int side, int v, const int* toff, const uint16_t* cold_before, int G,
+                                                const TileOrder& order) {
+  bool cold;
+  int k;
+  order.map(v, cold, k);
+  const int NT = order.NT;
+  int lo = 0, hi = G - 1;
+  while (lo < hi) {                       // first i with NT * class_before(i+1) > k
+    const int mid = (lo + hi) >> 1;
+    if (NT * class_before(toff, cold_before, cold, mid + 1) > k) hi = mid; else lo = mid + 1;
+  }
+  const int local = k - NT * class_before(toff, cold_before, cold, lo);
   const int Mi = toff[lo + 1] - toff[lo];
   WorkItem w;
   w.side = side;
