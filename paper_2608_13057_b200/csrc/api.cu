@@ -88,12 +88,11 @@ static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, 
   const uint8_t* blob = static_cast<const uint8_t*>(packed);
   const int sms = sm_count();
   if (sms <= 0) return TEMPO_ERR_CUDA;
-  CUtensorMap tmA1, tmA2, tmH, tmY;
+  CUtensorMap tmA1, tmA2, tmY;
   // a side that does not run still needs a well-formed map; point it at a buffer that exists
   if (!make_map(&tmA1, (run_mask & 1) ? a_q : h_q, s->M_cap, (run_mask & 1) ? s->d : s->f, 128)) return TEMPO_ERR_CUDA;
   if (!make_map(&tmA2, h_q, s->M_cap, s->f, 128)) return TEMPO_ERR_CUDA;
-  // stores: 32-row x 128-byte boxes of H (u8) and of Y (bf16 seen as bytes: 2d per row)
-  if (!make_map(&tmH, h_q, s->M_cap, s->f, 32)) return TEMPO_ERR_CUDA;
+  // Y stores: 32-row x 128-byte boxes (bf16 seen as bytes: 2d per row)
   if (!make_map(&tmY, (run_mask & 2) ? y : h_q, s->M_cap, (run_mask & 2) ? 2ull * s->d : s->f, 32)) return TEMPO_ERR_CUDA;
   FfnParams p{};
   p.side[0] = GemmSide{s->d / 128, L.J1, L.NT1, blob + L.off_w13, a_sf, blob + L.off_sf13};
@@ -113,9 +112,9 @@ static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, 
   p.done = p.ready ? p.ready + s->M_cap / 128 : nullptr;
   p.status = status;
   if (!use_pair_kernel(s))
-    return launch_ffn(tmA1, tmA2, tmH, tmY, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+    return launch_ffn(tmA1, tmA2, tmY, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
   PairMaps m;
-  m.a1 = tmA1; m.a2 = tmA2; m.h = tmH; m.y = tmY;
+  m.a1 = tmA1; m.a2 = tmA2; m.y = tmY;
   const size_t sf1_bytes = static_cast<size_t>(s->M_cap / 128) * L.J1 * 512, sf2_bytes = static_cast<size_t>(s->M_cap / 128) * L.J2 * 512;
   if (!make_flat_map(&m.w, blob, L.total, 128)) return TEMPO_ERR_CUDA;
   if (!make_flat_map(&m.sfb, blob, L.total, 8)) return TEMPO_ERR_CUDA;
@@ -343,10 +342,9 @@ int tempo_grouped_ffn_bf16(const tempo_shape* s, const void* a_bf16, const void*
   const uint8_t* blob = static_cast<const uint8_t*>(packed);
   const int sms = sm_count();
   if (sms <= 0) return TEMPO_ERR_CUDA;
-  CUtensorMap tmA1, tmA2, tmH, tmY;    // bf16 matrices seen as bytes: 2d / 2f per row
+  CUtensorMap tmA1, tmA2, tmY;    // bf16 matrices seen as bytes: 2d / 2f per row
   if (!make_map(&tmA1, a_bf16, s->M_cap, 2ull * s->d, 128)) return TEMPO_ERR_CUDA;
   if (!make_map(&tmA2, h_bf16, s->M_cap, 2ull * s->f, 128)) return TEMPO_ERR_CUDA;
-  if (!make_map(&tmH, h_bf16, s->M_cap, 2ull * s->f, 32)) return TEMPO_ERR_CUDA;
   if (!make_map(&tmY, y_bf16, s->M_cap, 2ull * s->d, 32)) return TEMPO_ERR_CUDA;
   FfnParams p{};
   p.side[0] = GemmSide{s->d / 64, 0, L.NT1, blob + L.off_w13, nullptr, nullptr};
@@ -363,7 +361,7 @@ int tempo_grouped_ffn_bf16(const tempo_shape* s, const void* a_bf16, const void*
   p.ready = static_cast<int32_t*>(workspace);
   p.done = p.ready + s->M_cap / 128;
   p.status = status;
-  return launch_ffn_bf16(tmA1, tmA2, tmH, tmY, p, sms, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK
+  return launch_ffn_bf16(tmA1, tmA2, tmY, p, sms, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK
                                                                                                          : TEMPO_ERR_CUDA;
 }
 

@@ -28,8 +28,7 @@
 //              to the MMA issuer at once, then the math (the pair shares the row maximum through
 //              shared memory).  Y leaves through swizzled staging in shared memory and TMA tensor
 //              stores; H leaves through ordinary 16-byte stores, because other CTAs wait for it and
-//              a TMA store queues behind the weight loads already issued for the next tile (tmH is
-//              not used by this kernel; the CTA-pair kernel takes the same four maps and uses it)
+//              a TMA store queues behind the weight loads already issued for the next tile
 // Scales are UE8M0 per 128 K-elements; the MMA takes one scale byte per row (A) and per column
 // (B) for each K=32 step, so the four steps of a K-block select the same byte (scale id kb % 4).
 //
@@ -51,7 +50,7 @@ constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 4
 template <bool kBf16>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
-           const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmY, const FfnParams p) {
+           const __grid_constant__ CUtensorMap tmY, const FfnParams p) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t s_full[kStages];
   __shared__ __align__(8) uint64_t s_empty[kStages];
@@ -463,23 +462,23 @@ size_t ffn_workspace_bytes(int M_cap) {
 }
 
 template <bool kBf16>
-static cudaError_t launch_ffn_t(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH,
-                                const CUtensorMap& tmY, const FfnParams& p, int num_sms, cudaStream_t stream) {
+static cudaError_t launch_ffn_t(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
+                                const FfnParams& p, int num_sms, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(ffn_kernel<kBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(kGemmSmemBytes));
   if (e != cudaSuccess) return e;
   const int grid = max(1, num_sms);   // one persistent CTA per SM; CTAs without work leave at once
-  return launch_pdl(ffn_kernel<kBf16>, dim3(grid), dim3(kGemmThreads), kGemmSmemBytes, stream, tmA1, tmA2, tmH, tmY, p);
+  return launch_pdl(ffn_kernel<kBf16>, dim3(grid), dim3(kGemmThreads), kGemmSmemBytes, stream, tmA1, tmA2, tmY, p);
 }
 
-cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH, const CUtensorMap& tmY,
+cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
                        const FfnParams& p, int num_sms, cudaStream_t stream) {
-  return launch_ffn_t<false>(tmA1, tmA2, tmH, tmY, p, num_sms, stream);
+  return launch_ffn_t<false>(tmA1, tmA2, tmY, p, num_sms, stream);
 }
 
-cudaError_t launch_ffn_bf16(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH,
-                            const CUtensorMap& tmY, const FfnParams& p, int num_sms, cudaStream_t stream) {
-  return launch_ffn_t<true>(tmA1, tmA2, tmH, tmY, p, num_sms, stream);
+cudaError_t launch_ffn_bf16(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
+                            const FfnParams& p, int num_sms, cudaStream_t stream) {
+  return launch_ffn_t<true>(tmA1, tmA2, tmY, p, num_sms, stream);
 }
 
 }  // namespace tempo

@@ -155,7 +155,7 @@ __device__ __forceinline__ PairItem decode_pair(int side, int x, const int* toff
 
 __global__ void __launch_bounds__(kPThreads, 1)
 ffn_pair_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
-                const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmY,
+                const __grid_constant__ CUtensorMap tmY,
                 const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmSfb,
                 const __grid_constant__ CUtensorMap tmSfa1, const __grid_constant__ CUtensorMap tmSfa2,
                 const FfnParams p, const PairRows pr) {
@@ -195,7 +195,6 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant_
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmSfb)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmSfa1)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmSfa2)) : "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmH)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmY)) : "memory");
   }
   if (warp == 1) {   // both CTAs of the pair take part in the allocation
@@ -292,8 +291,8 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant_
             }
           }
           if (!ok) break;
-          __threadfence();
-          asm volatile("fence.proxy.async;" ::: "memory");   // H was written through another proxy, TMA reads it
+          __threadfence_block();
+          asm volatile("fence.proxy.async;" ::: "memory");   // H was written by ordinary stores, TMA reads it
         }
         for (int kb = 0; kb < gs.Kb; ++kb) {
           if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
@@ -332,12 +331,12 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant_
           }
         }
         if (!ok) break;
+        __threadfence_block();
+        *s_dep = ++cleared;                      // tell the producer first, then do the bookkeeping
         if (atomicAdd(p.done + tau, 1) == p.side[1].NT - 1) {
           atomicExch(p.ready + tau, 0);
           atomicExch(p.done + tau, 0);
         }
-        __threadfence();
-        *s_dep = ++cleared;
       }
     }
   } else if (warp == 1) {
@@ -378,7 +377,8 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant_
   } else if (warp >= kPEpiWarp0) {
     // ------------------------------- epilogue --------------------------------------------------
     // As in the one-CTA kernel (two warps per tensor-memory lane quadrant, raw copy to registers,
-    // release, arithmetic, swizzled staging, TMA stores), on this CTA's own 128 rows.
+    // release, arithmetic, ordinary stores for H, swizzled staging + TMA stores for Y), on this
+    // CTA's own 128 rows.
     const int quad = warp & 3;
     const int half = (warp - kPEpiWarp0) >> 2;
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
@@ -440,11 +440,12 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant_
         }
 #define TEMPO_H(j) __uint_as_float(g[(j) >> 5][(j) & 31])
         s_amax[par][half][r_in_tile] = amax;
-        if (issuer) bulk_wait_read();
         pair_sync(pair_bar);
         amax = fmaxf(amax, s_amax[par][half ^ 1][r_in_tile]);
         const int eps = pow2_scale_exponent(amax);
         const float inv = pow2_neg(eps);
+        // ordinary stores for H, as in the one-CTA kernel (a TMA store would queue behind the loads)
+        uint4* dst = reinterpret_cast<uint4*>(p.h_q + static_cast<size_t>(row) * p.f + w.nt * 128 + half * 64);
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
           uint4 q;
@@ -452,19 +453,13 @@ ffn_pair_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant_
           q.y = cvt_e4m3x4(TEMPO_H(16 * v + 4) * inv, TEMPO_H(16 * v + 5) * inv, TEMPO_H(16 * v + 6) * inv, TEMPO_H(16 * v + 7) * inv);
           q.z = cvt_e4m3x4(TEMPO_H(16 * v + 8) * inv, TEMPO_H(16 * v + 9) * inv, TEMPO_H(16 * v + 10) * inv, TEMPO_H(16 * v + 11) * inv);
           q.w = cvt_e4m3x4(TEMPO_H(16 * v + 12) * inv, TEMPO_H(16 * v + 13) * inv, TEMPO_H(16 * v + 14) * inv, TEMPO_H(16 * v + 15) * inv);
-          st_shared_v4(my_line + (((half * 4 + v) ^ (lane & 7)) << 4), q);
+          dst[v] = q;
         }
 #undef TEMPO_H
         if (half == 0) p.h_sf[sf_index(row, w.nt, p.J_h)] = static_cast<uint8_t>(eps + 127);
-        fence_async_smem();
-        if (fused) __threadfence();
-        pair_sync(pair_bar);
-        if (issuer) {
-          tma_store_2d(&tmH, stage_buf, w.nt * 128, w.row0 + quad * 32);
-          bulk_commit();
-          if (fused) {
-            bulk_wait_all();
-            asm volatile("fence.proxy.async;" ::: "memory");
+        if (fused) {                                           // publish these 32 rows of the H block
+          pair_sync(pair_bar);
+          if (issuer) {
             __threadfence();
             atomicAdd(p.ready + (w.row0 >> 7), 1);
           }
@@ -549,7 +544,7 @@ cudaError_t launch_ffn_pair(const PairMaps& m, const FfnParams& p, const PairRow
   if (e != cudaSuccess) return e;
   if (resident < 1) return cudaErrorLaunchOutOfResources;
   if (static_cast<unsigned int>(2 * resident) < cfg.gridDim.x) cfg.gridDim = dim3(2 * resident);
-  return cudaLaunchKernelEx(&cfg, ffn_pair_kernel, m.a1, m.a2, m.h, m.y, m.w, m.sfb, m.sfa1, m.sfa2, p, pr);
+  return cudaLaunchKernelEx(&cfg, ffn_pair_kernel, m.a1, m.a2, m.y, m.w, m.sfb, m.sfa1, m.sfa2, p, pr);
 }
 
 }  // namespace tempo

@@ -106,9 +106,9 @@ struct FfnParams {
 };
 size_t ffn_workspace_bytes(int M_cap);
 // The bf16 variant: Kb counts 64-value K-blocks, the scale pointers and J_h are unused, h_q holds bf16.
-cudaError_t launch_ffn_bf16(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH,
-                            const CUtensorMap& tmY, const FfnParams& p, int num_sms, cudaStream_t stream);
-cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmH, const CUtensorMap& tmY,
+cudaError_t launch_ffn_bf16(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
+                            const FfnParams& p, int num_sms, cudaStream_t stream);
+cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
                        const FfnParams& p, int num_sms, cudaStream_t stream);
 
 
@@ -121,7 +121,7 @@ struct PairRows {
 };
 struct PairMaps {
   CUtensorMap a1, a2;    // activations of the two GEMMs, 128-row boxes, 128-byte swizzle
-  CUtensorMap h, y;      // stores, 32-row boxes
+  CUtensorMap y;         // Y stores, 32-row boxes
   CUtensorMap w, sfb;    // flat views of the packed blob: 128-row and 8-row boxes
   CUtensorMap sfa1, sfa2;  // flat views of the activation scale buffers: 4-row boxes
 };
