@@ -9,7 +9,7 @@ constexpr int kDispThreads = 1024;
 constexpr int kDispWarps = kDispThreads / 32;
 constexpr int kKeep = 4;           // 32-pair steps of a warp whose ids stay in registers between the passes
 constexpr int kMaxCluster = 8;     // portable cluster size
-constexpr int kPairsPerCta = 4096; // pairs per CTA before another CTA joins the cluster
+constexpr int kPairsPerCta = 1024; // pairs per CTA before another CTA joins the cluster
 
 // Lanes of the warp that hold the same expert id as this lane (e < 0: none).  One ballot per id
 // bit: a fixed, short latency, where __match_any_sync takes one round per distinct value.

@@ -130,7 +130,7 @@ cudaError_t launch_permute_pad_bf16(const PermuteParams& p, __nv_bfloat16* a, in
 cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t stream) {
   const long long warps = static_cast<long long>(p.M_cap) * ((p.d + 511) >> 9);
   long long blocks = (warps + kPermWarps - 1) / kPermWarps;
-  const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 8;   // 8 CTAs of 8 warps fill an SM
+  const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 6;   // 6 CTAs of 8 warps are resident per SM at 40 registers
   if (blocks > cap) blocks = cap;
   return launch_pdl(permute_pad_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(kPermWarps * 32), 0, stream, p);
 }
