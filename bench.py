@@ -34,8 +34,8 @@ NOMINAL_FP8_OVER_BF16 = 2.0             # dense fp8 peak = 2 x dense bf16 peak o
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel from the committed ncu
 # capture (profiles/), keyed by workload; None until a capture exists for that workload.
 NCU_TRAFFIC_BYTES = {
-    "cfg2": 394.98e6,          # profiles/ffn_kernel_cfg2_flat_decode.md (391.08 MB read + 3.9 MB written)
-    "cfg5-8-1024": 233.7e6,    # profiles/ffn_kernel_cfg5_G8_N1024_linear.md
+    "cfg2": 395.02e6,          # profiles/ffn_kernel_cfg2_flat_decode.md (391.08 MB read + 3.9 MB written)
+    "cfg5-8-1024": 231.6e6,    # profiles/ffn_kernel_cfg5_G8_N1024_linear.md
 }
 
 
