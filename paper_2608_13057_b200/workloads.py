@@ -298,20 +298,26 @@ def config5_point(G: int, N: int, seed: int = 4, d: int = 4096, f: int = 1536, w
                     np.arange(G, dtype=np.int32), x, seed, seed)
 
 
-def config5_skewed(G: int, N: int, seed: int = 4, d: int = 4096, f: int = 1536, with_x: bool = True) -> Workload:
-    """The (G, N) point with the same total rows G*N spread unevenly: instance i gets about
-    2*N*(i+1)/(G+1) rows (a linear ramp, mean N), k=1, w=1.  For the paper's remark that a grouped GEMM can
-    run faster under uniform per-slot loads at equal (G, N) (Section "Limitations", L5)."""
-    T = G * N
-    m = np.floor(2.0 * N * (np.arange(G) + 1) / (G + 1)).astype(np.int64)
-    m[-1] += T - int(m.sum())
+def config5_rows(rows, seed: int = 4, d: int = 4096, f: int = 1536, with_x: bool = True, name: str = "") -> Workload:
+    """One instance per entry of `rows`, that many rows each, k=1, w=1 (tokens of an instance are contiguous)."""
+    m = np.asarray(rows, dtype=np.int64)
+    G, T = len(m), int(m.sum())
     ids = np.repeat(np.arange(G, dtype=np.int32), m).reshape(T, 1)
     w = np.ones((T, 1), np.float32)
     rmap = np.arange(G, dtype=np.int32).reshape(G, 1)
     quota = m.astype(np.int32).reshape(G, 1)
-    x = draw_activations(seed * 1000003 + G * 8191 + N + 7, T, d) if with_x else None
-    return Workload(f"cfg5-skewed-G{G}-N{N}", T, 1, G, G, 1, d, f, T, ids, w, rmap, quota,
+    x = draw_activations(seed * 1000003 + G * 8191 + T + 7, T, d) if with_x else None
+    return Workload(name or f"cfg5-rows-G{G}-T{T}", T, 1, G, G, 1, d, f, T, ids, w, rmap, quota,
                     np.arange(G, dtype=np.int32), x, seed, seed)
+
+
+def config5_skewed(G: int, N: int, seed: int = 4, d: int = 4096, f: int = 1536, with_x: bool = True) -> Workload:
+    """The (G, N) point with the same total rows G*N spread unevenly: instance i gets about
+    2*N*(i+1)/(G+1) rows (a linear ramp, mean N), k=1, w=1.  For the paper's remark that a grouped GEMM can
+    run faster under uniform per-slot loads at equal (G, N) (Section "Limitations", L5)."""
+    m = np.floor(2.0 * N * (np.arange(G) + 1) / (G + 1)).astype(np.int64)
+    m[-1] += G * N - int(m.sum())
+    return config5_rows(m, seed, d, f, with_x, name=f"cfg5-skewed-G{G}-N{N}")
 
 
 def random_small(seed: int, T: int = 24, E: int = 6, k: int = 2, R_max: int = 3, d: int = 256, f: int = 256,

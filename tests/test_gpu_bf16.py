@@ -42,6 +42,7 @@ def _cases():
     yield W.config5_point(1, 40, d=256, f=256)
     yield W.config5_point(3, 129, d=384, f=640)           # two tiles per instance, K not a multiple of 256
     yield W.random_small(420, T=40, E=6, k=2, d=256, f=384)
+    yield W.config5_skewed(6, 200, d=256, f=384)          # cold (1-2 tiles) and hot (3 tiles) instances together
     yield W.random_small(421, T=40, n_valid=23)
 
 

@@ -40,6 +40,7 @@ def _cases():
     yield W.config5_point(3, 129, d=384, f=640)           # two M-tiles per instance: whole pairs
     yield W.config5_point(2, 300, d=512, f=256)           # three M-tiles: one whole pair and one half pair
     yield W.random_small(402, T=40, E=6, k=2, d=256, f=384)
+    yield W.config5_skewed(6, 200, d=256, f=384)          # 1, 1, 2, 2, 3, 3 tiles per instance
     yield W.config2()                                     # every instance a single M-tile
     yield W.config5_point(8, 512)                         # several pairs per instance, full-size d and f
 

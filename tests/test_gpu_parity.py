@@ -188,6 +188,7 @@ def _small_block_cases():
     yield W.config1()
     yield W.config5_point(1, 40, d=256, f=256)
     yield W.config5_point(3, 129, d=384, f=640)           # two tiles per instance, odd block counts
+    yield W.config5_skewed(6, 200, d=256, f=384)          # 1, 1, 2, 2, 3, 3 tiles: cold and hot instances in one batch
     for s in range(3):
         yield W.random_small(400 + s, T=40, E=6, k=2, d=256, f=384)
     yield W.random_small(410, T=40, n_valid=23)
@@ -307,6 +308,23 @@ def test_sweep_points_sampled(B, G, N):
     wl = W.config5_point(G, N)
     buf = _run_block(B, wl)
     _sampled_rows_check(B, wl, buf, rows_per_inst=2, n_tokens=8)
+
+
+def test_hot_and_cold_instances_dealt_together_elementwise(B):
+    """Two hot instances (4 M-tiles) and eight cold ones (1-2 M-tiles) with enough tiles on both sides of the FFN
+    (12 gate/up and 9 down tiles per M-tile) for a whole wave to be dealt from both lists: every row against the oracle."""
+    wl = W.config5_rows([500, 500, 130, 130, 130, 130, 60, 60, 60, 60], d=2304, f=1536)
+    buf = _run_block(B, wl)
+    ref = O.expert_block(wl, M_cap=buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    _check_permute(buf, ref)
+    m_pad = int(ref["m_pad"])
+    assert m_pad == 128 * 20
+    mx, mean = _err(to_np(buf.y)[:m_pad], ref["y"][:m_pad])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("Y", mx, mean)
+    mx, mean = _err(to_np(buf.out), ref["out"])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("out", mx, mean)
+    assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
 
 
 def test_skewed_sweep_point_sampled(B):
