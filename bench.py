@@ -267,7 +267,7 @@ def run_gpu(args):
                                buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair, buf.tile_inst, buf.m_pad,
                                buf.status)
         ev[i][1].record()
-        B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status)
+        B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status, pair_row=buf.pair_row)
         ev[i][2].record()
         B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y, buf.status,
                             buf.workspace)

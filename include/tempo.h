@@ -164,9 +164,15 @@ int tempo_count_dispatch_sampled(const tempo_shape* shape, const int32_t* topk_i
  * integer with max|block| <= 448 * 2^eps (0 for an all-zero block), round-to-nearest-even,
  * saturating; padding rows are zero codes with scale 1.  Rows >= m_pad are not written.
  *   in   x bf16 [T, d], row_pair, m_pad        out  a_q u8 [M_cap, d], a_sf u8 [tempo_sf_bytes(M_cap, d)]
+ *   pair_row (optional, may be NULL): step 1's pair -> row map.  With it, and when x is too large to
+ *   stay in L2 (T*d*2 > 48 MB), the kernel walks the TOKENS, quantises each row of x once and writes it
+ *   to the rows of all its local pairs, so x is read from HBM once however many local pairs a token has;
+ *   otherwise it walks the rows and gathers.  Same output bit for bit.  pair_row and row_pair must come
+ *   from the same step-1 call.
  */
 int tempo_permute_pad(const tempo_shape* shape, const void* x_bf16, const int32_t* row_pair,
-                      const int32_t* m_pad, void* a_q, uint8_t* a_sf, uint32_t* status, void* stream);
+                      const int32_t* pair_row, const int32_t* m_pad, void* a_q, uint8_t* a_sf,
+                      uint32_t* status, void* stream);
 
 /*
  * Step 3a: per instance GU = A * W13^T (fp8 x fp8 -> fp32 on the tensor cores, block scales applied

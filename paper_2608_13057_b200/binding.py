@@ -136,8 +136,9 @@ def tempo_count_dispatch_sampled(shape, topk_ids, n_valid, replica_map, table, s
            "tempo_count_dispatch_sampled")
 
 
-def tempo_permute_pad(shape, x_bf16, row_pair, m_pad, a_q, a_sf, status):
+def tempo_permute_pad(shape, x_bf16, row_pair, m_pad, a_q, a_sf, status, pair_row=None):
     _check(_lib.tempo_permute_pad(ctypes.byref(shape), _ptr(x_bf16, torch.bfloat16), _ptr(row_pair, torch.int32),
+                                  _ptr(pair_row, torch.int32),
                                   _ptr(m_pad, torch.int32), _ptr(a_q, torch.uint8), _ptr(a_sf, torch.uint8),
                                   _ptr(status, torch.int32), _stream()), "tempo_permute_pad")
 
@@ -261,7 +262,7 @@ class RankBuffers:
         tempo_count_dispatch(s, self.topk_ids, self.n_valid, self.replica_map, self.quota, self.cum_counts,
                              self.counts, self.inst_count, self.inst_off, self.pair_row, self.row_pair,
                              self.tile_inst, self.m_pad, self.status)
-        tempo_permute_pad(s, self.x, self.row_pair, self.m_pad, self.a_q, self.a_sf, self.status)
+        tempo_permute_pad(s, self.x, self.row_pair, self.m_pad, self.a_q, self.a_sf, self.status, pair_row=self.pair_row)
         tempo_grouped_ffn(s, self.a_q, self.a_sf, packed, self.inst_off, self.m_pad, self.h_q, self.h_sf, self.y,
                           self.status, self.workspace)
         tempo_unpermute_combine(s, self.y, self.pair_row, self.topk_w, self.n_valid, self.out, self.status)

@@ -247,12 +247,12 @@ int tempo_count_dispatch_sampled(const tempo_shape* s, const int32_t* topk_ids, 
   return launch_count_dispatch_sampled(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
 
-int tempo_permute_pad(const tempo_shape* s, const void* x_bf16, const int32_t* row_pair, const int32_t* m_pad,
-                      void* a_q, uint8_t* a_sf, uint32_t* status, void* stream) {
+int tempo_permute_pad(const tempo_shape* s, const void* x_bf16, const int32_t* row_pair, const int32_t* pair_row,
+                      const int32_t* m_pad, void* a_q, uint8_t* a_sf, uint32_t* status, void* stream) {
   const int rc = check_shape(s);
   if (rc != TEMPO_OK) return rc;
   if (!x_bf16 || !row_pair || !m_pad || !a_q || !a_sf || !status) return TEMPO_ERR_NULL;
-  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, m_pad,
+  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, s->T, pair_row, m_pad,
                   static_cast<uint8_t*>(a_q), a_sf};
   return launch_permute_pad(p, sm_count(), static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
@@ -327,7 +327,7 @@ int tempo_permute_pad_bf16(const tempo_shape* s, const void* x_bf16, const int32
   const int rc = check_shape(s);
   if (rc != TEMPO_OK) return rc;
   if (!x_bf16 || !row_pair || !m_pad || !a_bf16 || !status) return TEMPO_ERR_NULL;
-  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, m_pad, nullptr, nullptr};
+  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, s->T, nullptr, m_pad, nullptr, nullptr};
   return launch_permute_pad_bf16(p, static_cast<__nv_bfloat16*>(a_bf16), sm_count(), static_cast<cudaStream_t>(stream)) ==
                  cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }

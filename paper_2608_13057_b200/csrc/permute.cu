@@ -95,6 +95,116 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_kernel(const Perm
   }
 }
 
+// Token-major form.  Phase A: one warp per (token, 512-column chunk), two in flight: a lane loads its 32
+// bytes of x and (lanes below k) one pair -> row entry, the block maxima and codes are computed ONCE and
+// stored to the row of every local pair of the token - x is read from HBM once, and the row index and
+// the activations arrive together instead of one after the other.  Phase B: rows of the padded
+// layout that hold no pair are filled with zero codes and scale 1.
+struct TokItem {
+  int t, col, row;      // row: this lane's pair -> row entry (lanes >= k: -1)
+  bool live, in;
+  uint4 lo, hi;
+};
+
+__device__ __forceinline__ void tok_load(const PermuteParams& p, int t, int chunk, bool live, int lane, TokItem& it) {
+  it.live = live;
+  it.t = live ? t : 0;
+  it.col = live ? chunk * 512 + lane * 16 : 0;
+  it.in = live && it.col < p.d;
+  it.row = (live && lane < p.k) ? __ldg(p.pair_row + static_cast<size_t>(it.t) * p.k + lane) : -1;
+  it.lo = make_uint4(0, 0, 0, 0);
+  it.hi = make_uint4(0, 0, 0, 0);
+  if (it.in) {
+    const __nv_bfloat16* src = p.x + static_cast<size_t>(it.t) * p.d + it.col;
+    it.lo = __ldcs(reinterpret_cast<const uint4*>(src));
+    it.hi = __ldcs(reinterpret_cast<const uint4*>(src + 8));
+  }
+}
+
+__device__ __forceinline__ void tok_finish(const PermuteParams& p, const TokItem& it, int lane, int J, int m_pad) {
+  if (__ballot_sync(0xffffffffu, it.row >= 0) == 0) return;     // no local pair: nothing to write
+  const uint32_t w[8] = {it.lo.x, it.lo.y, it.lo.z, it.lo.w, it.hi.x, it.hi.y, it.hi.z, it.hi.w};
+  __nv_bfloat162 m2 = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[0]));
+#pragma unroll
+  for (int i = 1; i < 8; ++i) m2 = __hmax2(m2, __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[i])));
+  const uint32_t mbits = *reinterpret_cast<const uint32_t*>(&m2);
+  float amax = fmaxf(__uint_as_float(mbits << 16), __uint_as_float(mbits & 0xffff0000u));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+  amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
+  const int eps = pow2_scale_exponent(amax);
+  const float inv = pow2_neg(eps);
+  float v[16];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+  uint4 q;
+  q.x = cvt_e4m3x4(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv);
+  q.y = cvt_e4m3x4(v[4] * inv, v[5] * inv, v[6] * inv, v[7] * inv);
+  q.z = cvt_e4m3x4(v[8] * inv, v[9] * inv, v[10] * inv, v[11] * inv);
+  q.w = cvt_e4m3x4(v[12] * inv, v[13] * inv, v[14] * inv, v[15] * inv);
+  for (int s = 0; s < p.k; ++s) {
+    const int row = __shfl_sync(0xffffffffu, it.row, s);
+    if (row < 0 || row >= m_pad || !it.in) continue;            // row: warp-uniform
+    __stcs(reinterpret_cast<uint4*>(p.a_q + static_cast<size_t>(row) * p.d + it.col), q);
+    if ((lane & 7) == 0) p.a_sf[sf_index(row, it.col >> 7, J)] = static_cast<uint8_t>(eps + 127);
+  }
+}
+
+__global__ void __launch_bounds__(kPermWarps * 32) permute_tokens_kernel(const PermuteParams p) {
+  const int lane = threadIdx.x & 31;
+  const int chunks = (p.d + 511) >> 9;
+  const int J = ((p.d >> 7) + 3) >> 2;
+  pdl_trigger();
+  const long long S = static_cast<long long>(gridDim.x) * kPermWarps;
+  const long long g0 = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5);
+  pdl_wait();
+  // ---- phase A: tokens -----------------------------------------------------------------------
+  {
+    int t_a = static_cast<int>(g0 / chunks), ch_a = static_cast<int>(g0 % chunks);
+    int t_b = static_cast<int>((g0 + S) / chunks), ch_b = static_cast<int>((g0 + S) % chunks);
+    const int step_t = static_cast<int>((2 * S) / chunks), step_c = static_cast<int>((2 * S) % chunks);
+    TokItem a, b;
+    if (t_a < p.T) {
+      tok_load(p, t_a, ch_a, true, lane, a);                    // issued together with the m_pad read below
+      tok_load(p, t_b, ch_b, t_b < p.T, lane, b);
+    }
+    const int m_pad = min(*p.m_pad, p.M_cap);
+    while (t_a < p.T) {
+      tok_finish(p, a, lane, J, m_pad);
+      if (b.live) tok_finish(p, b, lane, J, m_pad);
+      t_a += step_t; ch_a += step_c;
+      if (ch_a >= chunks) { ch_a -= chunks; ++t_a; }
+      t_b += step_t; ch_b += step_c;
+      if (ch_b >= chunks) { ch_b -= chunks; ++t_b; }
+      if (t_a < p.T) {
+        tok_load(p, t_a, ch_a, true, lane, a);
+        tok_load(p, t_b, ch_b, t_b < p.T, lane, b);
+      }
+    }
+  }
+  // ---- phase B: rows without a pair ----------------------------------------------------------
+  // One warp per (group of 32 rows, 512-column chunk), so the fill spreads over the whole grid.
+  const int m_pad = min(*p.m_pad, p.M_cap);
+  const long long groups = (m_pad + 31) >> 5;
+  for (long long g = g0; g < groups * chunks; g += S) {
+    const int base = static_cast<int>(g / chunks) * 32;
+    const int col = static_cast<int>(g % chunks) * 512 + lane * 16;
+    const int r = base + lane;
+    const bool pad = r < m_pad && __ldg(p.row_pair + r) < 0;
+    uint32_t todo = __ballot_sync(0xffffffffu, pad);
+    if (col >= p.d) continue;
+    while (todo) {
+      const int row = base + __ffs(todo) - 1;
+      todo &= todo - 1;
+      __stcs(reinterpret_cast<uint4*>(p.a_q + static_cast<size_t>(row) * p.d + col), make_uint4(0, 0, 0, 0));
+      if ((lane & 7) == 0) p.a_sf[sf_index(row, col >> 7, J)] = 127;
+    }
+  }
+}
+
 // bf16 variant of step 2: the gathered rows stay bf16 (no quantiser); rows without a pair are zero.
 // One warp per (row, 512-byte chunk), 16 bytes per lane.
 __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_bf16_kernel(const PermuteParams p, __nv_bfloat16* a) {
@@ -127,7 +237,23 @@ cudaError_t launch_permute_pad_bf16(const PermuteParams& p, __nv_bfloat16* a, in
   return launch_pdl(permute_pad_bf16_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(kPermWarps * 32), 0, stream, p, a);
 }
 
+static cudaError_t launch_permute_tokens(const PermuteParams& p, int num_sms, cudaStream_t stream) {
+  const long long chunks = (p.d + 511) >> 9;
+  const long long warps = max(static_cast<long long>(p.T) * chunks, (static_cast<long long>(p.M_cap) / 32 + 1) * chunks);
+  long long blocks = (warps + 2 * kPermWarps - 1) / (2 * kPermWarps);        // two items per warp per trip
+  const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 6;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return launch_pdl(permute_tokens_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(kPermWarps * 32), 0, stream, p);
+}
+
 cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t stream) {
+  // Token-major pays when the rows of x no longer stay in L2 between the (up to k) gathers of a token:
+  // measured on B200, config 4 (x = 117 MB) 150 -> 100 us; with x = 34 MB (config 3) the gathers hit L2
+  // anyway and the row-major walk is 2 us faster.
+  constexpr size_t kTokenMajorBytes = 48u << 20;
+  if (p.pair_row != nullptr && static_cast<size_t>(p.T) * p.d * 2 > kTokenMajorBytes)
+    return launch_permute_tokens(p, num_sms, stream);
   const long long warps = static_cast<long long>(p.M_cap) * ((p.d + 511) >> 9);
   long long blocks = (warps + kPermWarps - 1) / kPermWarps;
   const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 6;   // 6 CTAs of 8 warps are resident per SM at 40 registers

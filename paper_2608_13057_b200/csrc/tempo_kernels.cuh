@@ -51,6 +51,8 @@ struct PermuteParams {
   int k, d, M_cap;
   const __nv_bfloat16* x;
   const int32_t* row_pair;
+  int T;                      // token rows (token-major form only)
+  const int32_t* pair_row;    // NULL: row-major form (gather per row); else token-major form (quantise once per token)
   const int32_t* m_pad;
   uint8_t* a_q;
   uint8_t* a_sf;

@@ -327,6 +327,30 @@ def test_hot_and_cold_instances_dealt_together_elementwise(B):
     assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
 
 
+def test_permute_by_rows_and_by_tokens_agree_bitwise(B):
+    """tempo_permute_pad without pair_row walks the rows and gathers; with it, and x beyond 48 MB, it walks the
+    tokens and quantises each row of x once.  Same bytes, and both equal the oracle (x here is 52 MB)."""
+    wl = W.random_small(431, T=8192, E=8, k=2, R_max=2, d=3200, f=128, n_valid=8000)
+    buf = B.RankBuffers.for_workload(wl, with_weights=False)
+    s = buf.shape
+    B.tempo_count_dispatch(s, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts, buf.counts,
+                           buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair, buf.tile_inst, buf.m_pad, buf.status)
+    outs = []
+    for pair_row in (None, buf.pair_row):
+        buf.a_q.fill_(0x55)
+        buf.a_sf.fill_(0x55)
+        B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status, pair_row=pair_row)
+        torch.cuda.synchronize()
+        m = int(buf.m_pad.item())
+        outs.append((buf.a_q[:m].clone(), sf_decode(to_np(buf.a_sf), buf.M_cap, buf.d)[:m].copy()))
+        assert torch.all(buf.a_q[m:] == 0x55)                  # rows >= m_pad are not written
+    assert torch.equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    ref = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, buf.M_cap)
+    assert m == int(ref["m_pad"]) and m > 0
+    a_q, a_s = O.permute_pad(wl.x, ref["row_pair"], ref["m_pad"], wl.k)
+    assert codes_equal_mod_signed_zero(to_np(outs[1][0]), a_q[:m]).all() and np.array_equal(outs[1][1], a_s[:m])
+
+
 def test_skewed_sweep_point_sampled(B):
     """Same totals as a sweep point, rows spread unevenly over the instances (227 ... 1824 rows)."""
     wl = W.config5_skewed(8, 1024)
