@@ -231,6 +231,31 @@ int tempo_unpermute_combine(const tempo_shape* shape, const void* y_bf16, const 
                             void* stream);
 
 /*
+ * Masked layout (the layout of the masked grouped GEMM the paper calibrates for decode, Section 2.1 and
+ * Appendix B): instance i owns the FIXED row range [i*max_m, (i+1)*max_m) of every padded buffer and uses
+ * its first inst_count[i] rows; nothing moves when the counts change from step to step.  max_m is a
+ * multiple of 128 with G_max*max_m <= M_cap (TEMPO_ERR_SHAPE otherwise).
+ *   tempo_count_dispatch_masked  as tempo_count_dispatch with inst_off[i] = i*max_m, m_pad = G_max*max_m,
+ *        tile_inst[tile] = i only for the ceil(inst_count[i]/128) tiles of instance i that hold rows (-1
+ *        elsewhere); pairs beyond max_m rows of an instance are dropped (pair_row = -1, TEMPO_STATUS_CAPACITY).
+ *   tempo_permute_pad_masked     step 2 for that layout: writes the rows of the tiles in use (rows with a pair,
+ *        zero rows up to the next tile boundary) and leaves unused tiles alone.
+ *   tempo_grouped_ffn_masked     step 3 (one kernel, as tempo_grouped_ffn) on the tiles in use only.
+ * Step 4 is tempo_unpermute_combine.  Results per row are those of the grouped layout bit for bit.
+ */
+int tempo_count_dispatch_masked(const tempo_shape* shape, int32_t max_m, const int32_t* topk_ids,
+                                const int32_t* n_valid, const int32_t* replica_map, const int32_t* quota,
+                                uint32_t* cum_counts, int32_t* counts, int32_t* inst_count, int32_t* inst_off,
+                                int32_t* pair_row, int32_t* row_pair, int32_t* tile_inst, int32_t* m_pad,
+                                uint32_t* status, void* stream);
+int tempo_permute_pad_masked(const tempo_shape* shape, const void* x_bf16, const int32_t* row_pair,
+                             const int32_t* pair_row, const int32_t* tile_inst, const int32_t* m_pad, void* a_q,
+                             uint8_t* a_sf, uint32_t* status, void* stream);
+int tempo_grouped_ffn_masked(const tempo_shape* shape, int32_t max_m, const void* a_q, const uint8_t* a_sf,
+                             const void* packed, const int32_t* inst_count, void* h_q, uint8_t* h_sf, void* y_bf16,
+                             uint32_t* status, void* workspace, void* stream);
+
+/*
  * bf16 variant of steps 2 and 3 (the paper calibrates a bf16 grouped GEMM beside the fp8 one and finds
  * the same two-regime shape with a later inflection: Section 2.1, Table "Fitted cost parameters").
  * No quantiser: the gathered rows stay bf16, both GEMMs multiply bf16 values with fp32 accumulation

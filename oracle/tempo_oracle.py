@@ -88,7 +88,11 @@ def replica_boundaries(n_e: int, slots, quotas, G_max: int, claimed: set):
     return valid, B, status
 
 
-def count_dispatch(topk_ids, n_valid, replica_map, quota, G_max, M_cap, cum_counts=None):
+def count_dispatch(topk_ids, n_valid, replica_map, quota, G_max, M_cap, cum_counts=None, max_m=None):
+    """max_m=None: instances follow each other, each padded to whole 128-row tiles (the grouped layout).
+    max_m=M (a multiple of 128): the MASKED layout of the grouped GEMM the paper calibrates ("fp8 masked
+    grouped GEMM", Appendix B): instance i owns the fixed row range [i*M, (i+1)*M) and only its first
+    inst_count[i] rows are in use; pairs beyond M rows of an instance are dropped (CAPACITY)."""
     ids = np.asarray(topk_ids, dtype=np.int64)
     T, k = ids.shape
     E, R = np.asarray(replica_map).shape
@@ -124,7 +128,12 @@ def count_dispatch(topk_ids, n_valid, replica_map, quota, G_max, M_cap, cum_coun
     # padded offsets in ascending slot id
     off = [0] * (G_max + 1)
     for i in range(G_max):
-        off[i + 1] = off[i] + TILE_M * ((m[i] + TILE_M - 1) // TILE_M)
+        if max_m is None:
+            off[i + 1] = off[i] + TILE_M * ((m[i] + TILE_M - 1) // TILE_M)
+        else:
+            off[i + 1] = off[i] + int(max_m)
+            if m[i] > max_m:
+                status |= STATUS_CAPACITY
     M_pad = off[G_max]
     if M_pad > M_cap:
         status |= STATUS_CAPACITY
@@ -141,18 +150,20 @@ def count_dispatch(topk_ids, n_valid, replica_map, quota, G_max, M_cap, cum_coun
             if j < B[e][r]:
                 if valid[e][r]:                   # (B only grows on valid columns, so this holds)
                     row = off[int(replica_map[e][r])] + (j - prev)
-                    if row < M_cap:
+                    if row < M_cap and (max_m is None or j - prev < max_m):
                         pair_row[p] = row
                         row_pair[row] = p
                 break
             prev = B[e][r]
 
     inst_off = np.minimum(np.array(off, dtype=np.int64), M_cap).astype(np.int32)
-    inst_count = np.array([max(0, min(m[i], M_cap - off[i])) for i in range(G_max)], dtype=np.int32)
+    inst_count = np.array([max(0, min(m[i], M_cap - off[i], m[i] if max_m is None else max_m))
+                           for i in range(G_max)], dtype=np.int32)
     m_pad = min(M_pad, M_cap)
     tile_inst = np.full(M_cap // TILE_M, -1, dtype=np.int32)
     for i in range(G_max):
-        for tau in range(inst_off[i] // TILE_M, inst_off[i + 1] // TILE_M):
+        used = inst_off[i + 1] if max_m is None else min(inst_off[i + 1], inst_off[i] + TILE_M * (-(-int(inst_count[i]) // TILE_M)))
+        for tau in range(inst_off[i] // TILE_M, used // TILE_M):
             tile_inst[tau] = i
 
     out = dict(counts=counts, inst_count=inst_count, inst_off=inst_off, pair_row=pair_row,
@@ -270,7 +281,7 @@ def expert_ffn(a_q, a_s, w13_q, w13_s, w2_q, w2_s):
     return h_q, h_s, Y
 
 
-def grouped_ffn(a_q, a_s, inst_off, inst_count, slot_weights, rows_only=None):
+def grouped_ffn(a_q, a_s, inst_off, inst_count, slot_weights, rows_only=None, masked=False):
     """slot_weights(i) -> (w13_q, w13_s, w2_q, w2_s) of instance slot i.
 
     Computes every padded row of every activated instance (pad rows are zero rows and give zeros).
@@ -281,6 +292,8 @@ def grouped_ffn(a_q, a_s, inst_off, inst_count, slot_weights, rows_only=None):
     h_q = h_s = y = None
     for i in range(G):
         lo, hi = int(inst_off[i]), int(inst_off[i + 1])
+        if masked:                                         # only the tiles that hold rows are computed
+            hi = min(hi, lo + TILE_M * (-(-int(inst_count[i]) // TILE_M)))
         if hi <= lo:
             continue
         w = slot_weights(i)
@@ -315,17 +328,18 @@ def combine(y, pair_row, topk_w, n_valid, T, k):
 # whole block
 # ----------------------------------------------------------------------------------------
 
-def expert_block(wl, M_cap=None, cum_counts=None):
-    """Runs all five steps on a workload object (fields as in the seeded generators)."""
+def expert_block(wl, M_cap=None, cum_counts=None, max_m=None):
+    """Runs all five steps on a workload object (fields as in the seeded generators).
+    max_m: the masked layout (see count_dispatch); rows outside the tiles in use are left zero."""
     M_cap = wl.M_cap if M_cap is None else M_cap
-    disp = count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, M_cap, cum_counts)
+    disp = count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, M_cap, cum_counts, max_m)
     a_q, a_s = permute_pad(wl.x, disp["row_pair"], disp["m_pad"], wl.k)
 
     def slot_weights(i):
         w = wl.expert_weights(int(wl.slot_expert[i]))
         return w.w13_q, w.w13_s, w.w2_q, w.w2_s
 
-    h_q, h_s, y = grouped_ffn(a_q, a_s, disp["inst_off"], disp["inst_count"], slot_weights)
+    h_q, h_s, y = grouped_ffn(a_q, a_s, disp["inst_off"], disp["inst_count"], slot_weights, masked=max_m is not None)
     if y is None:
         y = np.zeros((M_cap, wl.d), np.float32)
         h_q = np.zeros((M_cap, wl.f), np.uint8)

@@ -22,6 +22,7 @@ EXPORTS = (
     "tempo_packed_weight_bytes",
     "tempo_pack_weights", "tempo_count_dispatch", "tempo_count_dispatch_sampled", "tempo_permute_pad", "tempo_ffn_gate_up", "tempo_ffn_down",
     "tempo_grouped_ffn", "tempo_grouped_ffn_static", "tempo_unpermute_combine",
+    "tempo_count_dispatch_masked", "tempo_permute_pad_masked", "tempo_grouped_ffn_masked",
     "tempo_packed_weight_bytes_bf16", "tempo_pack_weights_bf16", "tempo_permute_pad_bf16", "tempo_grouped_ffn_bf16",
 )
 
@@ -182,6 +183,33 @@ def tempo_unpermute_combine(shape, y_bf16, pair_row, topk_w, n_valid, out_bf16, 
                                         _ptr(status, torch.int32), _stream()), "tempo_unpermute_combine")
 
 
+def tempo_count_dispatch_masked(shape, max_m, topk_ids, n_valid, replica_map, quota, cum_counts, counts, inst_count,
+                                inst_off, pair_row, row_pair, tile_inst, m_pad, status):
+    i32 = torch.int32
+    _check(_lib.tempo_count_dispatch_masked(ctypes.byref(shape), ctypes.c_int32(max_m), _ptr(topk_ids, i32),
+                                            _ptr(n_valid, i32), _ptr(replica_map, i32), _ptr(quota, i32),
+                                            _ptr(cum_counts, i32), _ptr(counts, i32), _ptr(inst_count, i32),
+                                            _ptr(inst_off, i32), _ptr(pair_row, i32), _ptr(row_pair, i32),
+                                            _ptr(tile_inst, i32), _ptr(m_pad, i32), _ptr(status, i32), _stream()),
+           "tempo_count_dispatch_masked")
+
+
+def tempo_permute_pad_masked(shape, x_bf16, row_pair, pair_row, tile_inst, m_pad, a_q, a_sf, status):
+    i32 = torch.int32
+    _check(_lib.tempo_permute_pad_masked(ctypes.byref(shape), _ptr(x_bf16, torch.bfloat16), _ptr(row_pair, i32),
+                                         _ptr(pair_row, i32), _ptr(tile_inst, i32), _ptr(m_pad, i32),
+                                         _ptr(a_q, torch.uint8), _ptr(a_sf, torch.uint8), _ptr(status, i32), _stream()),
+           "tempo_permute_pad_masked")
+
+
+def tempo_grouped_ffn_masked(shape, max_m, a_q, a_sf, packed, inst_count, h_q, h_sf, y_bf16, status, workspace):
+    _check(_lib.tempo_grouped_ffn_masked(ctypes.byref(shape), ctypes.c_int32(max_m), _ptr(a_q, torch.uint8),
+                                         _ptr(a_sf, torch.uint8), _ptr(packed, torch.uint8),
+                                         _ptr(inst_count, torch.int32), _ptr(h_q, torch.uint8), _ptr(h_sf, torch.uint8),
+                                         _ptr(y_bf16, torch.bfloat16), _ptr(status, torch.int32),
+                                         _ptr(workspace, torch.uint8), _stream()), "tempo_grouped_ffn_masked")
+
+
 def tempo_packed_weight_bytes_bf16(shape: TempoShape) -> int:
     out = ctypes.c_size_t(0)
     _check(_lib.tempo_packed_weight_bytes_bf16(ctypes.byref(shape), ctypes.byref(out)), "tempo_packed_weight_bytes_bf16")
@@ -265,6 +293,19 @@ class RankBuffers:
         tempo_permute_pad(s, self.x, self.row_pair, self.m_pad, self.a_q, self.a_sf, self.status, pair_row=self.pair_row)
         tempo_grouped_ffn(s, self.a_q, self.a_sf, packed, self.inst_off, self.m_pad, self.h_q, self.h_sf, self.y,
                           self.status, self.workspace)
+        tempo_unpermute_combine(s, self.y, self.pair_row, self.topk_w, self.n_valid, self.out, self.status)
+
+    def run_block_masked(self, max_m, packed=None):
+        """One pass of the block in the masked layout (instance i at rows [i*max_m, (i+1)*max_m))."""
+        s = self.shape
+        packed = self.packed if packed is None else packed
+        tempo_count_dispatch_masked(s, max_m, self.topk_ids, self.n_valid, self.replica_map, self.quota, self.cum_counts,
+                                    self.counts, self.inst_count, self.inst_off, self.pair_row, self.row_pair,
+                                    self.tile_inst, self.m_pad, self.status)
+        tempo_permute_pad_masked(s, self.x, self.row_pair, self.pair_row, self.tile_inst, self.m_pad, self.a_q, self.a_sf,
+                                 self.status)
+        tempo_grouped_ffn_masked(s, max_m, self.a_q, self.a_sf, packed, self.inst_count, self.h_q, self.h_sf, self.y,
+                                 self.status, self.workspace)
         tempo_unpermute_combine(s, self.y, self.pair_row, self.topk_w, self.n_valid, self.out, self.status)
 
     # ---- bf16 variant (separate activation / weight buffers, allocated on first use) ----

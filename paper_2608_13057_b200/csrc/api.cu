@@ -83,7 +83,8 @@ static int sm_count() {
 // run_mask bit 0: gate/up tiles, bit 1: down tiles.  Buffers a side does not use may be NULL.
 static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
                            const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y,
-                           uint32_t* status, void* workspace, cudaStream_t stream) {
+                           uint32_t* status, void* workspace, cudaStream_t stream, int max_m = 0,
+                           const int32_t* inst_count = nullptr) {
   const PackLayout L = pack_layout(s->G_max, s->d, s->f);
   const uint8_t* blob = static_cast<const uint8_t*>(packed);
   const int sms = sm_count();
@@ -105,6 +106,9 @@ static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, 
   p.J_h = L.J2;
   p.inst_off = inst_off;
   p.m_pad = m_pad;
+  p.stride_tiles = max_m / 128;
+  p.inst_count = inst_count;
+  if (max_m > 0 && use_pair_kernel(s)) return TEMPO_ERR_UNSUPPORTED;   // the pair kernel knows the grouped layout only
   p.h_q = static_cast<uint8_t*>(h_q);
   p.h_sf = h_sf;
   p.y = static_cast<__nv_bfloat16*>(y);
@@ -252,7 +256,7 @@ int tempo_permute_pad(const tempo_shape* s, const void* x_bf16, const int32_t* r
   const int rc = check_shape(s);
   if (rc != TEMPO_OK) return rc;
   if (!x_bf16 || !row_pair || !m_pad || !a_q || !a_sf || !status) return TEMPO_ERR_NULL;
-  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, s->T, pair_row, m_pad,
+  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, s->T, pair_row, nullptr, m_pad,
                   static_cast<uint8_t*>(a_q), a_sf};
   return launch_permute_pad(p, sm_count(), static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
@@ -304,6 +308,50 @@ int tempo_grouped_ffn_static(const tempo_shape* s, const void* a_q, const uint8_
                          static_cast<cudaStream_t>(stream));
 }
 
+// ---- masked layout ------------------------------------------------------------------------------------
+static int check_masked(const tempo_shape* s, int32_t max_m) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (max_m <= 0 || max_m % 128 != 0) return TEMPO_ERR_SHAPE;
+  if (static_cast<long long>(s->G_max) * max_m > s->M_cap) return TEMPO_ERR_SHAPE;
+  return TEMPO_OK;
+}
+
+int tempo_count_dispatch_masked(const tempo_shape* s, int32_t max_m, const int32_t* topk_ids, const int32_t* n_valid,
+                                const int32_t* replica_map, const int32_t* quota, uint32_t* cum_counts,
+                                int32_t* counts, int32_t* inst_count, int32_t* inst_off, int32_t* pair_row,
+                                int32_t* row_pair, int32_t* tile_inst, int32_t* m_pad, uint32_t* status, void* stream) {
+  const int rc = check_masked(s, max_m);
+  if (rc != TEMPO_OK) return rc;
+  if (!topk_ids || !replica_map || !quota || !counts || !inst_count || !inst_off || !pair_row || !row_pair ||
+      !tile_inst || !m_pad || !status)
+    return TEMPO_ERR_NULL;
+  DispatchParams p{s->T, s->k, s->E, s->G_max, s->R_max, s->M_cap, topk_ids, n_valid, replica_map, quota,
+                   cum_counts, counts, inst_count, inst_off, pair_row, row_pair, tile_inst, m_pad, status, max_m};
+  return launch_count_dispatch(p, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+int tempo_permute_pad_masked(const tempo_shape* s, const void* x_bf16, const int32_t* row_pair, const int32_t* pair_row,
+                             const int32_t* tile_inst, const int32_t* m_pad, void* a_q, uint8_t* a_sf,
+                             uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!x_bf16 || !row_pair || !pair_row || !tile_inst || !m_pad || !a_q || !a_sf || !status) return TEMPO_ERR_NULL;
+  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, s->T, pair_row, tile_inst,
+                  m_pad, static_cast<uint8_t*>(a_q), a_sf};
+  return launch_permute_pad(p, sm_count(), static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+int tempo_grouped_ffn_masked(const tempo_shape* s, int32_t max_m, const void* a_q, const uint8_t* a_sf,
+                             const void* packed, const int32_t* inst_count, void* h_q, uint8_t* h_sf, void* y_bf16,
+                             uint32_t* status, void* workspace, void* stream) {
+  const int rc = check_masked(s, max_m);
+  if (rc != TEMPO_OK) return rc;
+  if (!a_q || !a_sf || !packed || !inst_count || !h_q || !h_sf || !y_bf16 || !status || !workspace) return TEMPO_ERR_NULL;
+  return launch_ffn_host(3, s, a_q, a_sf, packed, nullptr, nullptr, h_q, h_sf, y_bf16, status, workspace,
+                         static_cast<cudaStream_t>(stream), max_m, inst_count);
+}
+
 // ---- bf16 variant of steps 2 and 3 -------------------------------------------------------------------
 int tempo_packed_weight_bytes_bf16(const tempo_shape* s, size_t* bytes) {
   if (bytes == nullptr) return TEMPO_ERR_NULL;
@@ -327,7 +375,7 @@ int tempo_permute_pad_bf16(const tempo_shape* s, const void* x_bf16, const int32
   const int rc = check_shape(s);
   if (rc != TEMPO_OK) return rc;
   if (!x_bf16 || !row_pair || !m_pad || !a_bf16 || !status) return TEMPO_ERR_NULL;
-  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, s->T, nullptr, m_pad, nullptr, nullptr};
+  PermuteParams p{s->k, s->d, s->M_cap, static_cast<const __nv_bfloat16*>(x_bf16), row_pair, s->T, nullptr, nullptr, m_pad, nullptr, nullptr};
   return launch_permute_pad_bf16(p, static_cast<__nv_bfloat16*>(a_bf16), sm_count(), static_cast<cudaStream_t>(stream)) ==
                  cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }

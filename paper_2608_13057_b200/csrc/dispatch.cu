@@ -163,7 +163,12 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
   __syncthreads();
 
   // ---- padded offsets: exclusive scan of 128*ceil(m/128) in ascending slot id (warp 0) -------
-  if (warp == 0) {
+  // (masked layout: instance i simply starts at row i * max_m)
+  if (p.max_m > 0) {
+    for (int i = tid; i <= G; i += kDispThreads) off[i] = i * p.max_m;
+    for (int i = tid; i < G; i += kDispThreads)
+      if (m_inst[i] > p.max_m && cta == 0) my_status |= TEMPO_STATUS_CAPACITY;
+  } else if (warp == 0) {
     if (lane == 0) s_carry = 0;
     __syncwarp();
     for (int base = 0; base < G; base += 32) {
@@ -193,7 +198,7 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
     }
     for (int i = tid; i <= G; i += kDispThreads) {
       p.inst_off[i] = min(off[i], p.M_cap);
-      if (i < G) p.inst_count[i] = max(0, min(m_inst[i], p.M_cap - off[i]));
+      if (i < G) p.inst_count[i] = max(0, min(min(m_inst[i], p.M_cap - off[i]), p.max_m > 0 ? p.max_m : m_inst[i]));
     }
     for (int tau = tid; tau < p.M_cap / kTileM; tau += kDispThreads) {
       const int row = tau * kTileM;
@@ -205,6 +210,8 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
           if (off[mid + 1] > row) hi = mid; else lo = mid + 1;
         }
         inst = lo;
+        // masked layout: only the tiles that hold rows belong to the instance
+        if (p.max_m > 0 && row - off[lo] >= ((min(m_inst[lo], p.max_m) + kTileM - 1) / kTileM) * kTileM) inst = -1;
       }
       p.tile_inst[tau] = inst;
     }
@@ -238,7 +245,7 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
           const int B = bnd[e * R + r];
           if (j < B) {                                           // B only grows on valid columns
             const int cand = off[rmap_s[e * R + r]] + (j - prev);
-            if (cand < p.M_cap) row = cand;
+            if (cand < p.M_cap && (p.max_m == 0 || j - prev < p.max_m)) row = cand;
             break;
           }
           prev = B;

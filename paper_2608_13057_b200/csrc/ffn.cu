@@ -88,15 +88,34 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   pdl_wait();
-  const int m_pad = max(0, min(*p.m_pad, p.M_cap)) & ~(kTileM - 1);
-  const int m_tiles = m_pad / kTileM;
+  const int stride = p.stride_tiles;
+  if (stride > 0) {
+    // masked layout: M-tiles in use before each instance, from the row counts (warp 0 scans)
+    if (warp == 0) {
+      int carry = 0;
+      for (int base = 0; base < G; base += 32) {
+        const int i = base + lane;
+        const int c = i < G ? min(stride, (max(0, p.inst_count[i]) + kTileM - 1) / kTileM) : 0;
+        int incl = c;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += v;
+        }
+        if (i < G) s_toff[i] = carry + incl - c;
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      if (lane == 0) s_toff[G] = carry;
+    }
+  } else {
+    const int m_pad_c = max(0, min(*p.m_pad, p.M_cap)) & ~(kTileM - 1);
+    for (int i = tid; i <= G; i += kGemmThreads) s_toff[i] = max(0, min(p.inst_off[i], m_pad_c)) >> 7;
+  }
+  __syncthreads();
+  const int m_tiles = s_toff[G];
   const int n1 = (p.run_mask & 1) ? m_tiles * p.side[0].NT : 0;
   const int n2 = (p.run_mask & 2) ? m_tiles * p.side[1].NT : 0;
   const bool fused = p.run_mask == 3;
   const int Kb1 = p.side[0].Kb, Kb2 = p.side[1].Kb;
-
-  for (int i = tid; i <= G; i += kGemmThreads) s_toff[i] = max(0, min(p.inst_off[i], m_pad)) >> 7;
-  __syncthreads();
   if (warp == 0) {   // cold[i] = M-tiles of cold instances before instance i
     int carry = 0;
     for (int base = 0; base < G; base += 32) {
@@ -129,7 +148,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       int side, x;
       while (ok && it.next(side, x)) {
         const GemmSide& gs = p.side[side];
-        const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2);
+        const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2, stride);
         const uint8_t* sfb_src = gs.sfb + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.JK * kSfbBytes;
         const uint8_t* b_src = gs.wt + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.Kb * kBBytes;
         const bool stream_b = w.m_tiles <= 2;
@@ -156,7 +175,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       int side, x;
       while (ok && it.next(side, x)) {
         const GemmSide& gs = p.side[side];
-        const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2);
+        const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2, stride);
         const uint8_t* sfa_src = gs.sfa + static_cast<size_t>(w.row0 >> 7) * gs.JK * kSfaBytes;
         const CUtensorMap* tm = side == 0 ? &tmA1 : &tmA2;
         if (side == 1 && fused) {
@@ -203,7 +222,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       bool ok = true;
       while (ok && it.next(side, x)) {
         if (side == 0) continue;
-        const WorkItem w = decode_item(1, x, s_toff, s_cold, G, order2);
+        const WorkItem w = decode_item(1, x, s_toff, s_cold, G, order2, stride);
         const int tau = w.row0 >> 7;
         unsigned long long t0 = 0;
         for (uint32_t spin = 0; ld_acquire(p.ready + tau) < want; ++spin) {
@@ -285,7 +304,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
     int side, x;
     while (it.next(side, x)) {
-      const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2);
+      const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2, stride);
       const int row = w.row0 + r_in_tile;
       // Both warps of a pair must take the same way out: they vote on the outcome of the wait.
       const bool ok = mbar_wait(smem_u32(&s_acc_full), acc_phase, s_abort);

@@ -216,7 +216,7 @@ __device__ __forceinline__ int class_before(const int* toff, const uint16_t* col
 }
 
 __device__ __forceinline__ WorkItem decode_item(int side, int v, const int* toff, const uint16_t* cold_before, int G,
-                                                const TileOrder& order) {
+                                                const TileOrder& order, int stride_tiles = 0) {
   bool cold;
   int k;
   order.map(v, cold, k);
@@ -232,7 +232,7 @@ __device__ __forceinline__ WorkItem decode_item(int side, int v, const int* toff
   w.side = side;
   w.inst = lo;
   w.nt = local / Mi;
-  w.row0 = (toff[lo] + local % Mi) * kTileM;
+  w.row0 = ((stride_tiles > 0 ? lo * stride_tiles : toff[lo]) + local % Mi) * kTileM;   // masked layout: fixed stride
   w.m_tiles = Mi;
   return w;
 }

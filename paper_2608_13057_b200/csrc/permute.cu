@@ -193,7 +193,8 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_tokens_kernel(const P
     const int base = static_cast<int>(g / chunks) * 32;
     const int col = static_cast<int>(g % chunks) * 512 + lane * 16;
     const int r = base + lane;
-    const bool pad = r < m_pad && __ldg(p.row_pair + r) < 0;
+    bool pad = r < m_pad && __ldg(p.row_pair + r) < 0;
+    if (pad && p.tile_inst != nullptr) pad = __ldg(p.tile_inst + (r >> 7)) >= 0;   // masked layout: used tiles only
     uint32_t todo = __ballot_sync(0xffffffffu, pad);
     if (col >= p.d) continue;
     while (todo) {
@@ -252,8 +253,8 @@ cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t
   // measured on B200, config 4 (x = 117 MB) 150 -> 100 us; with x = 34 MB (config 3) the gathers hit L2
   // anyway and the row-major walk is 2 us faster.
   constexpr size_t kTokenMajorBytes = 48u << 20;
-  if (p.pair_row != nullptr && static_cast<size_t>(p.T) * p.d * 2 > kTokenMajorBytes)
-    return launch_permute_tokens(p, num_sms, stream);
+  if (p.pair_row != nullptr && (p.tile_inst != nullptr || static_cast<size_t>(p.T) * p.d * 2 > kTokenMajorBytes))
+    return launch_permute_tokens(p, num_sms, stream);                 // the masked layout always walks the tokens
   const long long warps = static_cast<long long>(p.M_cap) * ((p.d + 511) >> 9);
   long long blocks = (warps + kPermWarps - 1) / kPermWarps;
   const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 6;   // 6 CTAs of 8 warps are resident per SM at 40 registers

@@ -22,6 +22,7 @@ struct DispatchParams {
   int32_t* tile_inst;
   int32_t* m_pad;
   uint32_t* status;
+  int max_m;   // 0: instances follow each other in whole tiles; M > 0: masked layout, instance i owns rows [i*M, (i+1)*M)
 };
 size_t dispatch_smem_bytes(int E, int R, int G);
 
@@ -53,6 +54,7 @@ struct PermuteParams {
   const int32_t* row_pair;
   int T;                      // token rows (token-major form only)
   const int32_t* pair_row;    // NULL: row-major form (gather per row); else token-major form (quantise once per token)
+  const int32_t* tile_inst;   // masked layout only (else NULL): tiles with -1 hold no rows and are left alone
   const int32_t* m_pad;
   uint8_t* a_q;
   uint8_t* a_sf;
@@ -99,6 +101,10 @@ struct FfnParams {
   int J_h;               // scale atoms along f of the H buffer
   const int32_t* inst_off;
   const int32_t* m_pad;
+  // masked layout (stride_tiles > 0): instance i owns the M-tiles [i*stride_tiles, (i+1)*stride_tiles) and
+  // uses the first ceil(inst_count[i]/128) of them; inst_off and m_pad are not read
+  int stride_tiles;
+  const int32_t* inst_count;
   uint8_t* h_q;
   uint8_t* h_sf;
   __nv_bfloat16* y;
