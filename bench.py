@@ -226,12 +226,13 @@ def run_gpu(args):
 
     wl = make_workload(args.workload, rank)
     st = workload_stats(wl)
-    buf = B.RankBuffers.for_workload(wl)
+    max_m = args.max_m                                 # > 0: the masked layout, instance i at rows [i*max_m, (i+1)*max_m)
+    buf = B.RankBuffers.for_workload(wl, M_cap=wl.G_max * max_m if max_m else None)
     weight_bytes_all = buf.packed.numel()
     n_pools = max(2, math.ceil((1 << 30) / max(weight_bytes_all, 1)))
     n_pools = min(n_pools, 64)
     pools = [buf.packed] + [buf.packed.clone() for _ in range(n_pools - 1)]
-    graphs = _capture_graphs(torch, buf, pools)
+    graphs = _capture_graphs(torch, buf, pools, (lambda packed: buf.run_block_masked(max_m, packed=packed)) if max_m else None)
     K, Wm = args.steps, args.warmup
 
     def barrier():
@@ -263,14 +264,25 @@ def run_gpu(args):
     for i in range(Kb):
         blob = pools[i % n_pools]
         ev[i][0].record()
-        B.tempo_count_dispatch(s, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts, buf.counts,
-                               buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair, buf.tile_inst, buf.m_pad,
-                               buf.status)
-        ev[i][1].record()
-        B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status, pair_row=buf.pair_row)
-        ev[i][2].record()
-        B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y, buf.status,
-                            buf.workspace)
+        if max_m:
+            B.tempo_count_dispatch_masked(s, max_m, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts,
+                                          buf.counts, buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair,
+                                          buf.tile_inst, buf.m_pad, buf.status)
+            ev[i][1].record()
+            B.tempo_permute_pad_masked(s, buf.x, buf.row_pair, buf.pair_row, buf.tile_inst, buf.m_pad, buf.a_q, buf.a_sf,
+                                       buf.status)
+            ev[i][2].record()
+            B.tempo_grouped_ffn_masked(s, max_m, buf.a_q, buf.a_sf, blob, buf.inst_count, buf.h_q, buf.h_sf, buf.y,
+                                       buf.status, buf.workspace)
+        else:
+            B.tempo_count_dispatch(s, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts, buf.counts,
+                                   buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair, buf.tile_inst, buf.m_pad,
+                                   buf.status)
+            ev[i][1].record()
+            B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status, pair_row=buf.pair_row)
+            ev[i][2].record()
+            B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
+                                buf.status, buf.workspace)
         ev[i][3].record()
         B.tempo_unpermute_combine(s, buf.y, buf.pair_row, buf.topk_w, buf.n_valid, buf.out, buf.status)
         ev[i][4].record()
@@ -341,6 +353,7 @@ def run_gpu(args):
         "data": "synthetic",
         "config": {"workload": args.workload, "T": wl.T, "top_k": wl.k, "E": wl.E, "d": wl.d, "f": wl.f,
                    "G_act": st["G_act"], "N_local": st["N_local"], "M_pad": st["M_pad"],
+                   "layout": f"masked, max_m={max_m}" if max_m else "grouped",
                    "l2": f"weights rotate through {n_pools} copies ({n_pools * weight_bytes_all / 1e9:.2f} GB >> L2)",
                    "parallelism": f"{world} independent rank(s), no collective"},
         "block_us": us_step, "tokens_per_s": st["n_valid"] * world / (us_step * 1e-6),
@@ -454,6 +467,7 @@ def main():
     ap.add_argument("--sweep-N", default="")
     ap.add_argument("--replays", type=int, default=30)
     ap.add_argument("--variant", default="fp8", choices=["fp8", "bf16"], help="--sweep only: which steps 2 and 3")
+    ap.add_argument("--max-m", type=int, default=0, help="> 0: run the block in the masked layout with this row stride")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
