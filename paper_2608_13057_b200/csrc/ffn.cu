@@ -211,7 +211,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     }
   } else if (warp == 3) {
     // ------------------------------- dependency scout -----------------------------------------
-    // Runs ahead through this CTA's down tiles: waits (bounded) until the four epilogue warps of
+    // Runs ahead through this CTA's down tiles: waits (bounded) until the four epilogue warp pairs of
     // every gate/up tile of the tile's 128 rows have published their H rows, then tells the
     // activation producer through s_dep.  The last down tile of an M-tile to get here puts the
     // two global counters back to zero, so the workspace is clean when the kernel ends.
