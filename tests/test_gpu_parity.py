@@ -352,6 +352,24 @@ def test_permute_by_rows_and_by_tokens_agree_bitwise(B, n_valid):
     assert codes_equal_mod_signed_zero(to_np(outs[1][0]), a_q[:m]).all() and np.array_equal(outs[1][1], a_s[:m])
 
 
+def test_many_instances_elementwise(B):
+    """300 instance slots (the prefix scans of the FFN kernel run over ten 32-slot groups): empty, one-tile,
+    two-tile and four-tile instances mixed, every row against the oracle."""
+    rng = np.random.default_rng(77)
+    rows = rng.choice([0, 1, 37, 128, 129, 200, 300, 450], size=300, p=[0.1, 0.1, 0.3, 0.1, 0.1, 0.1, 0.1, 0.1])
+    wl = W.config5_rows(rows.tolist(), d=128, f=256)
+    buf = _run_block(B, wl)
+    ref = O.expert_block(wl, M_cap=buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    _check_permute(buf, ref)
+    m_pad = int(ref["m_pad"])
+    mx, mean = _err(to_np(buf.y)[:m_pad], ref["y"][:m_pad])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("Y", mx, mean)
+    mx, mean = _err(to_np(buf.out), ref["out"])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("out", mx, mean)
+    assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
+
+
 def test_skewed_sweep_point_sampled(B):
     """Same totals as a sweep point, rows spread unevenly over the instances (227 ... 1824 rows)."""
     wl = W.config5_skewed(8, 1024)
