@@ -370,6 +370,35 @@ def test_many_instances_elementwise(B):
     assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
 
 
+def test_limits_of_the_shape_elementwise(B):
+    """The documented maxima at once: 1024 experts, 1024 instance slots (most of them empty or tiny), d = f = 128."""
+    rng = np.random.default_rng(78)
+    rows = rng.choice([0, 0, 0, 1, 2, 5, 130], size=1024)
+    wl = W.config5_rows(rows.tolist(), d=128, f=128)
+    assert wl.E == 1024 and wl.G_max == 1024
+    buf = _run_block(B, wl)
+    ref = O.expert_block(wl, M_cap=buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    _check_permute(buf, ref)
+    m_pad = int(ref["m_pad"])
+    mx, mean = _err(to_np(buf.y)[:m_pad], ref["y"][:m_pad])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("Y", mx, mean)
+    mx, mean = _err(to_np(buf.out), ref["out"])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("out", mx, mean)
+    assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
+
+
+def test_top_k_32_elementwise(B):
+    """k at its documented maximum: 32 slots per token, 40 experts, every expert local."""
+    wl = W.random_small(460, T=24, E=40, k=32, R_max=1, d=128, f=128)
+    buf = _run_block(B, wl)
+    ref = O.expert_block(wl, M_cap=buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    _check_permute(buf, ref)
+    mx, mean = _err(to_np(buf.out), ref["out"])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("out", mx, mean)
+
+
 def test_skewed_sweep_point_sampled(B):
     """Same totals as a sweep point, rows spread unevenly over the instances (227 ... 1824 rows)."""
     wl = W.config5_skewed(8, 1024)
