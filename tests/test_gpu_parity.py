@@ -446,6 +446,22 @@ def test_graph_replay_matches_eager_launches(B):
     ref = O.expert_block(wl, M_cap=buf.M_cap)
     mx, mean = _err(to_np(buf.out), ref["out"])
     assert mx <= MAX_TOL and mean <= MEAN_TOL
+    # bench.py's chains: several consecutive steps in ONE graph, each step's first kernel launched
+    # programmatically behind the previous step's last one, n_valid changing between the steps
+    nv_a, nv_b = buf.n_valid.clone(), torch.full_like(buf.n_valid, 200)
+    chain = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(chain):
+        for i in range(6):
+            buf.n_valid.copy_(nv_b if i % 2 == 0 else nv_a)
+            buf.run_block(packed=other if i % 2 else buf.packed)
+    for t in (buf.pair_row, buf.a_q, buf.h_q, buf.y, buf.out):
+        t.zero_()
+    chain.replay()
+    chain.replay()
+    torch.cuda.synchronize()
+    for a, b in zip(eager, (buf.pair_row, buf.a_q, buf.h_q, buf.y, buf.out)):   # the last step ran with all rows live
+        assert torch.equal(a, b)
+    assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
 
 
 def test_bounded_wait_reports_timeout_and_the_context_stays_usable(B):
