@@ -464,6 +464,30 @@ def test_graph_replay_matches_eager_launches(B):
     assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
 
 
+def test_consecutive_steps_with_different_inputs_do_not_mix(B):
+    """The fused FFN hands H from CTA to CTA through counters; a down tile that started before its H block was
+    visible would read the previous step's block.  Consecutive steps therefore get different activations and the
+    last one is compared bit for bit with an eager run, many times over."""
+    wl = W.config2()
+    buf = _run_block(B, wl)
+    want = (buf.h_q.clone(), buf.y.clone(), buf.out.clone())
+    xa = buf.x.clone()
+    xb = (buf.x.float() * -1.5 + 0.25).to(torch.bfloat16)
+    other = buf.packed.clone()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for i in range(6):
+            buf.x.copy_(xb if i % 2 == 0 else xa)
+            buf.run_block(packed=other if i % 2 else buf.packed)
+    for _ in range(40):
+        buf.h_q.zero_()
+        buf.y.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(want[0], buf.h_q) and torch.equal(want[1], buf.y) and torch.equal(want[2], buf.out)
+    assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
+
+
 def test_bounded_wait_reports_timeout_and_the_context_stays_usable(B):
     """Failure detection without a fault: the down tiles wait for H-ready counters that nothing will
     complete (the workspace is poisoned on the host), the wait gives up after its one-second limit,
