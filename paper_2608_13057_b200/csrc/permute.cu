@@ -28,9 +28,14 @@ __device__ __forceinline__ void perm_load(const PermuteParams& p, int row, int c
   it.hi = make_uint4(0, 0, 0, 0);
 }
 
-__device__ __forceinline__ void perm_gather(const PermuteParams& p, PermItem& it) {
+// Token of a pair: a shift when k is a power of two (kshift >= 0), a division otherwise.
+__device__ __forceinline__ int pair_token(int pair, int k, int kshift) { return kshift >= 0 ? pair >> kshift : pair / k; }
+
+__device__ __forceinline__ int shift_of(int k) { return (k & (k - 1)) == 0 ? __ffs(k) - 1 : -1; }
+
+__device__ __forceinline__ void perm_gather(const PermuteParams& p, PermItem& it, int kshift) {
   if (it.in && it.pair >= 0) {
-    const __nv_bfloat16* src = p.x + static_cast<size_t>(it.pair / p.k) * p.d + it.col;
+    const __nv_bfloat16* src = p.x + static_cast<size_t>(pair_token(it.pair, p.k, kshift)) * p.d + it.col;
     it.lo = __ldcs(reinterpret_cast<const uint4*>(src));
     it.hi = __ldcs(reinterpret_cast<const uint4*>(src + 8));
   }
@@ -70,6 +75,7 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_kernel(const Perm
   const int lane = threadIdx.x & 31;
   const int chunks = (p.d + 511) >> 9;
   const int J = ((p.d >> 7) + 3) >> 2;
+  const int kshift = shift_of(p.k);
   pdl_trigger();
   pdl_wait();
   const int m_pad = min(*p.m_pad, p.M_cap);
@@ -84,8 +90,8 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_kernel(const Perm
     PermItem a, b;
     perm_load(p, row_a, ch_a, true, lane, a);
     perm_load(p, row_b, ch_b, row_b < m_pad, lane, b);
-    perm_gather(p, a);
-    perm_gather(p, b);
+    perm_gather(p, a, kshift);
+    perm_gather(p, b, kshift);
     perm_finish(p, a, lane, J);
     if (b.live) perm_finish(p, b, lane, J);
     row_a += step_r; ch_a += step_c;
