@@ -45,8 +45,10 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
   __shared__ int32_t s_carry;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  pdl_trigger();
+  // The next kernel's CTAs are let in only once the previous step has finished: released earlier they sit
+  // resident through that step's tail and cost it time (0.6 us per step on a decode-sized batch).
   pdl_wait();
+  pdl_trigger();
   int nv = p.T;
   if (p.n_valid != nullptr) nv = max(0, min(*p.n_valid, p.T));
   const int P = nv * p.k;                     // live pairs

@@ -212,6 +212,46 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_tokens_kernel(const P
   }
 }
 
+// One-wave form of the token-major walk, for batches small enough that every item gets a warp of its own
+// (decode-sized): warps [0, T * chunks) take one (token, chunk) each, the warps after them one
+// (group of kFillRows rows, chunk) of the zero fill, so nothing queues behind anything else and the kernel
+// lasts one index + activation latency instead of the two or three round trips of a grid-stride walk
+// (config 2: 5.5 -> 2.7 us from the end of the dispatch).  The next kernel is released after the wait: let in
+// earlier, its CTAs sit resident through the previous step's tail, which cost more than their prologue saves.
+constexpr int kFillRows = 16;
+
+__global__ void __launch_bounds__(kPermWarps * 32) permute_wave_kernel(const PermuteParams p) {
+  const int lane = threadIdx.x & 31;
+  const int chunks = (p.d + 511) >> 9;
+  const int J = ((p.d >> 7) + 3) >> 2;
+  const long long w = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5);
+  const long long n_tok = static_cast<long long>(p.T) * chunks;
+  pdl_wait();
+  pdl_trigger();
+  if (w < n_tok) {
+    TokItem a;
+    tok_load(p, static_cast<int>(w / chunks), static_cast<int>(w % chunks), true, lane, a);
+    const int m_pad = min(*p.m_pad, p.M_cap);
+    tok_finish(p, a, lane, J, m_pad);
+    return;
+  }
+  const long long g = w - n_tok;
+  const int base = static_cast<int>(g / chunks) * kFillRows;
+  const int col = static_cast<int>(g % chunks) * 512 + lane * 16;
+  if (base >= p.M_cap) return;
+  const int r = base + lane;
+  const int pair = (lane < kFillRows && r < p.M_cap) ? __ldg(p.row_pair + r) : 0;
+  const int m_pad = min(*p.m_pad, p.M_cap);
+  uint32_t todo = __ballot_sync(0xffffffffu, lane < kFillRows && r < m_pad && pair < 0);
+  if (col >= p.d) return;
+  while (todo) {
+    const int row = base + __ffs(todo) - 1;
+    todo &= todo - 1;
+    __stcs(reinterpret_cast<uint4*>(p.a_q + static_cast<size_t>(row) * p.d + col), make_uint4(0, 0, 0, 0));
+    if ((lane & 7) == 0) p.a_sf[sf_index(row, col >> 7, J)] = 127;
+  }
+}
+
 // bf16 variant of step 2: the gathered rows stay bf16 (no quantiser); rows without a pair are zero.
 // One warp per (row, 512-byte chunk), 16 bytes per lane.
 __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_bf16_kernel(const PermuteParams p, __nv_bfloat16* a) {
@@ -259,6 +299,14 @@ cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t
   // measured on B200, config 4 (x = 117 MB) 150 -> 100 us; with x = 34 MB (config 3) the gathers hit L2
   // anyway and the row-major walk is 2 us faster.
   constexpr size_t kTokenMajorBytes = 48u << 20;
+  if (p.pair_row != nullptr && p.tile_inst == nullptr) {
+    // a warp per item, all of them resident at once (4 CTAs per SM leave room beside the dispatch cluster)
+    const long long chunks = (p.d + 511) >> 9;
+    const long long warps = (static_cast<long long>(p.T) + (p.M_cap + kFillRows - 1) / kFillRows) * chunks;
+    const long long blocks = max(1LL, (warps + kPermWarps - 1) / kPermWarps);
+    if (blocks <= static_cast<long long>(num_sms > 0 ? num_sms : 148) * 4)
+      return launch_pdl(permute_wave_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(kPermWarps * 32), 0, stream, p);
+  }
   if (p.pair_row != nullptr && (p.tile_inst != nullptr || static_cast<size_t>(p.T) * p.d * 2 > kTokenMajorBytes))
     return launch_permute_tokens(p, num_sms, stream);                 // the masked layout always walks the tokens
   const long long warps = static_cast<long long>(p.M_cap) * ((p.d + 511) >> 9);
