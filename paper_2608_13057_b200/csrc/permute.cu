@@ -240,9 +240,11 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_wave_kernel(const Per
   const int col = static_cast<int>(g % chunks) * 512 + lane * 16;
   if (base >= p.M_cap) return;
   const int r = base + lane;
-  const int pair = (lane < kFillRows && r < p.M_cap) ? __ldg(p.row_pair + r) : 0;
+  const bool mine = lane < kFillRows && r < p.M_cap;
+  const int pair = mine ? __ldg(p.row_pair + r) : 0;
+  const int inst = (mine && p.tile_inst != nullptr) ? __ldg(p.tile_inst + (r >> 7)) : 0;   // masked layout: used tiles only
   const int m_pad = min(*p.m_pad, p.M_cap);
-  uint32_t todo = __ballot_sync(0xffffffffu, lane < kFillRows && r < m_pad && pair < 0);
+  uint32_t todo = __ballot_sync(0xffffffffu, mine && r < m_pad && pair < 0 && inst >= 0);
   if (col >= p.d) return;
   while (todo) {
     const int row = base + __ffs(todo) - 1;
@@ -299,7 +301,7 @@ cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t
   // measured on B200, config 4 (x = 117 MB) 150 -> 100 us; with x = 34 MB (config 3) the gathers hit L2
   // anyway and the row-major walk is 2 us faster.
   constexpr size_t kTokenMajorBytes = 48u << 20;
-  if (p.pair_row != nullptr && p.tile_inst == nullptr) {
+  if (p.pair_row != nullptr) {
     // a warp per item, all of them resident at once (4 CTAs per SM leave room beside the dispatch cluster)
     const long long chunks = (p.d + 511) >> 9;
     const long long warps = (static_cast<long long>(p.T) + (p.M_cap + kFillRows - 1) / kFillRows) * chunks;
