@@ -349,15 +349,64 @@ def run_gpu(args):
             h_out[j].copy_(b.out, non_blocking=True)
             ev_out[j].record(s_out)
 
-    Ke = min(K, 500)
+    # The same pipeline captured once: a graph of `ce` consecutive steps over the three streams (every step's
+    # copies are nodes of the graph), so the host issues one launch per `ce` steps and its timing drops out.
+    def capture_e2e(ce):
+        g = torch.cuda.CUDAGraph()
+        gi = [torch.cuda.Event() for _ in range(ce)]
+        gc = [torch.cuda.Event() for _ in range(ce)]
+        go = [torch.cuda.Event() for _ in range(ce)]
+        with torch.cuda.graph(g):
+            cur = torch.cuda.current_stream()
+            s_in.wait_stream(cur)
+            s_out.wait_stream(cur)
+            for i in range(ce):
+                b = sets[i & 1][0]
+                with torch.cuda.stream(s_in):
+                    if i >= 2:
+                        s_in.wait_event(gc[i - 2])     # this set's previous step has read its inputs
+                    b.topk_ids.copy_(h_ids, non_blocking=True)
+                    b.topk_w.copy_(h_w, non_blocking=True)
+                    b.x.copy_(h_x, non_blocking=True)
+                    gi[i].record(s_in)
+                cur.wait_event(gi[i])
+                if i >= 2:
+                    cur.wait_event(go[i - 2])          # and its previous result has left
+                if max_m:
+                    b.run_block_masked(max_m, packed=pools[i % n_pools])
+                else:
+                    b.run_block(packed=pools[i % n_pools])
+                gc[i].record(cur)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(gc[i])
+                    h_out[i & 1].copy_(b.out, non_blocking=True)
+                    go[i].record(s_out)
+            cur.wait_stream(s_in)
+            cur.wait_stream(s_out)
+        return g
+
+    Ke = min(K, 480)
+    ce = 2 * n_pools * max(1, 24 // n_pools)               # steps per captured graph (even: the buffer sets alternate)
     for i in range(min(Wm, 5) + 1):
         e2e_step(i)
     barrier()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    f0.record(s_in)
-    for i in range(Ke):
-        e2e_step(i)
-    f1.record(s_out)
+    if Ke >= ce:
+        g_e2e = capture_e2e(ce)
+        g_e2e.replay()
+        barrier()
+        Ke = (Ke // ce) * ce
+        f0.record()
+        for _ in range(Ke // ce):
+            g_e2e.replay()
+        f1.record()
+        e2e_mode = f"{ce} steps per CUDA graph, copies included"
+    else:
+        f0.record(s_in)
+        for i in range(Ke):
+            e2e_step(i)
+        f1.record(s_out)
+        e2e_mode = "launched step by step"
     barrier()
     ms_e2e = f0.elapsed_time(f1) / Ke
     e2e_ok = bool(torch.equal(h_out[0], h_out[1]) and torch.equal(h_out[0], buf.out.cpu()))
@@ -409,7 +458,8 @@ def run_gpu(args):
         "kernel_us": kern_us, "gpu_launches": 4 * K, "device_status": status,
         "roofline": roof, "clocks": clocks,
         "e2e": {"value": ms_e2e_max * 1e3 / units, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "pipeline": "two buffer sets, copy-in / compute / copy-out streams", "results_identical": e2e_ok},
+                "pipeline": "two buffer sets, copy-in / compute / copy-out streams; " + e2e_mode, "steps": Ke,
+                "results_identical": e2e_ok},
     }
     if world == 1 and not args.no_cpu_baseline:
         v, sample = oracle_sample_us_per_block(wl, budget_s=12.0)
