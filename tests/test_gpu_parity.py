@@ -352,6 +352,40 @@ def test_permute_by_rows_and_by_tokens_agree_bitwise(B, n_valid):
     assert codes_equal_mod_signed_zero(to_np(outs[1][0]), a_q[:m]).all() and np.array_equal(outs[1][1], a_s[:m])
 
 
+def _small_permute_cases():
+    yield W.config1()
+    yield W.config2(n_valid=200)
+    yield W.config5_point(3, 129, d=384, f=640)           # d below one 512-column chunk
+    yield W.random_small(432, T=40, E=6, k=3, d=640, f=128, n_valid=23)   # k not a power of two, ragged last chunk
+    yield W.random_small(433, T=1, E=4, k=2, d=256, f=128)
+    yield W.random_small(434, T=16, E=4, k=2, d=256, f=128, n_valid=0)
+
+
+@pytest.mark.parametrize("wl", list(_small_permute_cases()), ids=lambda w: w.name)
+def test_permute_of_a_decode_sized_batch_agrees_with_the_row_walk_bitwise(B, wl):
+    """With pair_row and a batch small enough for one warp per item, tempo_permute_pad runs its one-wave kernel;
+    without pair_row it walks the rows.  Same bytes in rows below m_pad, nothing written above, both equal the oracle."""
+    buf = B.RankBuffers.for_workload(wl, with_weights=False)
+    s = buf.shape
+    B.tempo_count_dispatch(s, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts, buf.counts,
+                           buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair, buf.tile_inst, buf.m_pad, buf.status)
+    outs = []
+    for pair_row in (None, buf.pair_row):
+        buf.a_q.fill_(0x55)
+        buf.a_sf.fill_(0x55)
+        B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status, pair_row=pair_row)
+        torch.cuda.synchronize()
+        m = int(buf.m_pad.item())
+        outs.append((buf.a_q[:m].clone(), sf_decode(to_np(buf.a_sf), buf.M_cap, buf.d)[:m].copy()))
+        assert torch.all(buf.a_q[m:] == 0x55)
+    assert torch.equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    ref = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, buf.M_cap)
+    assert m == int(ref["m_pad"])
+    a_q, a_s = O.permute_pad(wl.x, ref["row_pair"], ref["m_pad"], wl.k)
+    assert codes_equal_mod_signed_zero(to_np(outs[1][0]), a_q[:m]).all() and np.array_equal(outs[1][1], a_s[:m])
+    assert int(buf.status.item()) == 0
+
+
 def test_many_instances_elementwise(B):
     """300 instance slots (the prefix scans of the FFN kernel run over ten 32-slot groups): empty, one-tile,
     two-tile and four-tile instances mixed, every row against the oracle."""
