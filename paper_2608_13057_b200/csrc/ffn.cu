@@ -93,6 +93,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     // masked layout: M-tiles in use before each instance, from the row counts (warp 0 scans)
     if (warp == 0) {
       int carry = 0;
+#pragma unroll 1
       for (int base = 0; base < G; base += 32) {
         const int i = base + lane;
         const int c = i < G ? min(stride, (max(0, p.inst_count[i]) + kTileM - 1) / kTileM) : 0;
@@ -108,6 +109,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     }
   } else {
     const int m_pad_c = max(0, min(*p.m_pad, p.M_cap)) & ~(kTileM - 1);
+#pragma unroll 1
     for (int i = tid; i <= G; i += kGemmThreads) s_toff[i] = max(0, min(p.inst_off[i], m_pad_c)) >> 7;
   }
   __syncthreads();
@@ -118,6 +120,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   const int Kb1 = p.side[0].Kb, Kb2 = p.side[1].Kb;
   if (warp == 0) {   // cold[i] = M-tiles of cold instances before instance i
     int carry = 0;
+#pragma unroll 1
     for (int base = 0; base < G; base += 32) {
       const int i = base + lane;
       const int Mi = i < G ? s_toff[i + 1] - s_toff[i] : 0;
@@ -152,6 +155,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         const uint8_t* sfb_src = gs.sfb + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.JK * kSfbBytes;
         const uint8_t* b_src = gs.wt + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.Kb * kBBytes;
         const bool stream_b = w.m_tiles <= 2;
+#pragma unroll 1
         for (int kb = 0; kb < gs.Kb; ++kb) {
           if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
           const uint32_t full = smem_u32(&s_full[stage]);
@@ -197,6 +201,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
           __threadfence_block();
           asm volatile("fence.proxy.async;" ::: "memory");
         }
+#pragma unroll 1
         for (int kb = 0; kb < gs.Kb; ++kb) {
           if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
           const uint32_t full = smem_u32(&s_full[stage]);
@@ -253,6 +258,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         const int Kb = p.side[side].Kb;
         if (!mbar_wait(smem_u32(&s_acc_empty), acc_phase ^ 1u, s_abort)) break;
         tc_fence_after();
+#pragma unroll 1
         for (int kb = 0; kb < Kb; ++kb) {
           if (!mbar_wait(smem_u32(&s_full[stage]), phase, s_abort)) { ok = false; break; }
           tc_fence_after();
