@@ -242,7 +242,8 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_wave_kernel(const Per
   const int r = base + lane;
   const bool mine = lane < kFillRows && r < p.M_cap;
   const int pair = mine ? __ldg(p.row_pair + r) : 0;
-  const int inst = (mine && p.tile_inst != nullptr) ? __ldg(p.tile_inst + (r >> 7)) : 0;   // masked layout: used tiles only
+  // masked layout: used tiles only (tile_inst has M_cap / 128 entries)
+  const int inst = (mine && p.tile_inst != nullptr && (r >> 7) < p.M_cap / kTileM) ? __ldg(p.tile_inst + (r >> 7)) : 0;
   const int m_pad = min(*p.m_pad, p.M_cap);
   uint32_t todo = __ballot_sync(0xffffffffu, mine && r < m_pad && pair < 0 && inst >= 0);
   if (col >= p.d) return;

@@ -74,6 +74,26 @@ def test_masked_block_matches_oracle_elementwise(B, wl, max_m):
     assert int(buf.workspace.max().item()) == 0
 
 
+def test_masked_layout_with_spare_capacity(B):
+    """M_cap above G_max * max_m: the tiles above the last instance's range hold nothing and are left alone."""
+    wl = W.random_small(452, T=40, E=6, k=2, d=256, f=384)
+    max_m = 128
+    M_cap = wl.G_max * max_m + 256
+    buf = B.RankBuffers.for_workload(wl, M_cap=M_cap)
+    buf.a_q.fill_(0x55)
+    buf.run_block_masked(max_m)
+    torch.cuda.synchronize()
+    ref = O.expert_block(wl, M_cap=M_cap, max_m=max_m)
+    got = dispatch_outputs(buf)
+    for key in ("counts", "inst_count", "inst_off", "pair_row", "row_pair", "tile_inst"):
+        assert np.array_equal(got[key], ref[key]), key
+    assert got["m_pad"] == int(ref["m_pad"]) and got["status"] == int(ref["status"]) == 0
+    assert torch.all(buf.a_q[wl.G_max * max_m:] == 0x55)
+    out = to_np(buf.out)
+    mx, mean = _err(out[:wl.n_valid], ref["out"][:wl.n_valid])
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("out", mx, mean)
+
+
 def test_masked_and_grouped_layouts_give_the_same_output_bitwise(B):
     wl = W.config2()
     grouped = B.RankBuffers.for_workload(wl)
