@@ -54,6 +54,8 @@ def make_workload(name: str, rank: int = 0):
         return W.config1(seed=0 + 101 * rank)
     if name == "cfg2":
         return W.config2(seed=1 + 101 * rank)
+    if name.startswith("cfg2-T"):                      # cfg2-T512: the same rank with another decode batch size
+        return W.config2(seed=1 + 101 * rank, T=int(name[6:]))
     if name.startswith("cfg3-"):
         return W.config3(name[5:].replace("-", "_"), seed=2 + 101 * rank)
     if name == "cfg4":

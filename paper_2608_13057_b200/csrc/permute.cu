@@ -224,34 +224,37 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_wave_kernel(const Per
   const int lane = threadIdx.x & 31;
   const int chunks = (p.d + 511) >> 9;
   const int J = ((p.d >> 7) + 3) >> 2;
-  const long long w = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5);
+  const long long S = static_cast<long long>(gridDim.x) * kPermWarps;
   const long long n_tok = static_cast<long long>(p.T) * chunks;
+  const long long n_all = n_tok + static_cast<long long>((p.M_cap + kFillRows - 1) / kFillRows) * chunks;
   pdl_wait();
   pdl_trigger();
-  if (w < n_tok) {
-    TokItem a;
-    tok_load(p, static_cast<int>(w / chunks), static_cast<int>(w % chunks), true, lane, a);
+  // (the grid holds a warp per item up to 4 CTAs per SM; beyond that a warp takes two or three items in turn)
+  for (long long w = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5); w < n_all; w += S) {
+    if (w < n_tok) {
+      TokItem a;
+      tok_load(p, static_cast<int>(w / chunks), static_cast<int>(w % chunks), true, lane, a);
+      const int m_pad = min(*p.m_pad, p.M_cap);
+      tok_finish(p, a, lane, J, m_pad);
+      continue;
+    }
+    const long long g = w - n_tok;
+    const int base = static_cast<int>(g / chunks) * kFillRows;
+    const int col = static_cast<int>(g % chunks) * 512 + lane * 16;
+    const int r = base + lane;
+    const bool mine = lane < kFillRows && r < p.M_cap;
+    const int pair = mine ? __ldg(p.row_pair + r) : 0;
+    // masked layout: used tiles only (tile_inst has M_cap / 128 entries)
+    const int inst = (mine && p.tile_inst != nullptr && (r >> 7) < p.M_cap / kTileM) ? __ldg(p.tile_inst + (r >> 7)) : 0;
     const int m_pad = min(*p.m_pad, p.M_cap);
-    tok_finish(p, a, lane, J, m_pad);
-    return;
-  }
-  const long long g = w - n_tok;
-  const int base = static_cast<int>(g / chunks) * kFillRows;
-  const int col = static_cast<int>(g % chunks) * 512 + lane * 16;
-  if (base >= p.M_cap) return;
-  const int r = base + lane;
-  const bool mine = lane < kFillRows && r < p.M_cap;
-  const int pair = mine ? __ldg(p.row_pair + r) : 0;
-  // masked layout: used tiles only (tile_inst has M_cap / 128 entries)
-  const int inst = (mine && p.tile_inst != nullptr && (r >> 7) < p.M_cap / kTileM) ? __ldg(p.tile_inst + (r >> 7)) : 0;
-  const int m_pad = min(*p.m_pad, p.M_cap);
-  uint32_t todo = __ballot_sync(0xffffffffu, mine && r < m_pad && pair < 0 && inst >= 0);
-  if (col >= p.d) return;
-  while (todo) {
-    const int row = base + __ffs(todo) - 1;
-    todo &= todo - 1;
-    __stcs(reinterpret_cast<uint4*>(p.a_q + static_cast<size_t>(row) * p.d + col), make_uint4(0, 0, 0, 0));
-    if ((lane & 7) == 0) p.a_sf[sf_index(row, col >> 7, J)] = 127;
+    uint32_t todo = __ballot_sync(0xffffffffu, mine && r < m_pad && pair < 0 && inst >= 0);
+    if (col >= p.d) continue;
+    while (todo) {
+      const int row = base + __ffs(todo) - 1;
+      todo &= todo - 1;
+      __stcs(reinterpret_cast<uint4*>(p.a_q + static_cast<size_t>(row) * p.d + col), make_uint4(0, 0, 0, 0));
+      if ((lane & 7) == 0) p.a_sf[sf_index(row, col >> 7, J)] = 127;
+    }
   }
 }
 
@@ -303,12 +306,17 @@ cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t
   // anyway and the row-major walk is 2 us faster.
   constexpr size_t kTokenMajorBytes = 48u << 20;
   if (p.pair_row != nullptr) {
-    // a warp per item, all of them resident at once (4 CTAs per SM leave room beside the dispatch cluster)
+    // a warp per item, all of them resident at once (4 CTAs per SM leave room beside the dispatch cluster);
+    // larger batches keep that grid and give a warp several items
     const long long chunks = (p.d + 511) >> 9;
     const long long warps = (static_cast<long long>(p.T) + (p.M_cap + kFillRows - 1) / kFillRows) * chunks;
     const long long blocks = max(1LL, (warps + kPermWarps - 1) / kPermWarps);
-    if (blocks <= static_cast<long long>(num_sms > 0 ? num_sms : 148) * 4)
-      return launch_pdl(permute_wave_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(kPermWarps * 32), 0, stream, p);
+    const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 4;
+    // up to six items per warp it still beats the row walk (measured: T = 1024 -1.2 us, T = 2048 -3 us per block;
+    // at T = 4096, ten items per warp, it is 1.4 us behind)
+    if (blocks <= 6 * cap)
+      return launch_pdl(permute_wave_kernel, dim3(static_cast<unsigned int>(min(blocks, cap))), dim3(kPermWarps * 32), 0,
+                        stream, p);
   }
   if (p.pair_row != nullptr && (p.tile_inst != nullptr || static_cast<size_t>(p.T) * p.d * 2 > kTokenMajorBytes))
     return launch_permute_tokens(p, num_sms, stream);                 // the masked layout always walks the tokens

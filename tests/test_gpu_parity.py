@@ -359,6 +359,7 @@ def _small_permute_cases():
     yield W.random_small(432, T=40, E=6, k=3, d=640, f=128, n_valid=23)   # k not a power of two, ragged last chunk
     yield W.random_small(433, T=1, E=4, k=2, d=256, f=128)
     yield W.random_small(434, T=16, E=4, k=2, d=256, f=128, n_valid=0)
+    yield W.config2(T=1024)                               # three items per warp in the one-wave kernel
 
 
 @pytest.mark.parametrize("wl", list(_small_permute_cases()), ids=lambda w: w.name)
