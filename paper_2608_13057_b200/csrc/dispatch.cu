@@ -86,19 +86,29 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
 
   // ---- pass 1: warp histograms -------------------------------------------------------------
   int kept[kKeep];                            // ids of the first kKeep steps, reused by pass 2
+  // the ids of those steps are requested together, so a warp with several steps pays the latency once
 #pragma unroll
-  for (int i = 0; i < kKeep; ++i) kept[i] = -1;
+  for (int i = 0; i < kKeep; ++i) {
+    const int pidx = w_begin + 32 * i + lane;
+    int e = -1;
+    if (pidx < w_end) {
+      e = __ldg(p.topk_ids + pidx);
+      if (e < 0 || e >= E) { my_status |= TEMPO_STATUS_BAD_ID; e = -1; }
+    }
+    kept[i] = e;
+  }
   {
     int step = 0;
     for (int base = w_begin; base < w_end; base += 32, ++step) {
       const int pidx = base + lane;
       int e = -1;
-      if (pidx < w_end) {
+      if (step < kKeep) {
+#pragma unroll
+        for (int i = 0; i < kKeep; ++i) if (i == step) e = kept[i];
+      } else if (pidx < w_end) {
         e = __ldg(p.topk_ids + pidx);
         if (e < 0 || e >= E) { my_status |= TEMPO_STATUS_BAD_ID; e = -1; }
       }
-#pragma unroll
-      for (int i = 0; i < kKeep; ++i) if (i == step) kept[i] = e;
       const uint32_t same = same_expert_mask(e, id_bits);
       if (e >= 0 && lane == __ffs(same) - 1) hist[warp * E + e] += __popc(same);
       __syncwarp();
