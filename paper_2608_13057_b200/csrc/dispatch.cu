@@ -249,8 +249,10 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
       p.tile_inst[tau] = inst;
     }
   }
-  // every CTA has pre-filled its share of row_pair, and nobody reads a neighbour's totals any more
-  cluster.sync();
+  // Nobody reads a neighbour's totals any more (a CTA must not run ahead and exit while they are being read).
+  // This barrier orders no memory - the pre-fill of row_pair was ordered before the scatters below by the
+  // cluster barrier after pass 1 - so it is taken without the release/acquire fences of cluster.sync().
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;\n\tbarrier.cluster.wait.aligned;" ::: "memory");
 
   // ---- pass 2: stable ranks -> replica -> row -------------------------------------------------
   int step = 0;
