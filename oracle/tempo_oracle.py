@@ -28,8 +28,11 @@ Pins (tests/test_oracle_*.py): numpy.bincount and stable argsort for counts and 
 separately written sort-and-cut brute force for replica assignment, exact quota and
 bijection invariants, torch's CPU float8_e4m3fn cast for the code rounding, half-ulp error
 bounds and idempotence for the quantiser, torch fp32 dense SwiGLU MLP for the FFN, split
-invariance and linearity for the whole block; for the bf16 variant torch's CPU bfloat16 cast
-and the same dense-MLP and split-invariance checks.  No function here is "parity unpinned".
+invariance and linearity for the whole block, and the layer as Section 2.1 defines it written
+token by token with no layout (out[t] = sum_s w[t,s] * FFN_e(x[t]) over the experts held here,
+k > 1, remote experts, dead rows, stale quota rows); for the bf16 variant torch's CPU bfloat16
+cast and the same dense-MLP, per-token and split-invariance checks.  No function here is
+"parity unpinned".
 """
 from __future__ import annotations
 

@@ -158,3 +158,108 @@ def test_combine_is_a_weighted_gather_sum():
     assert np.allclose(out[0], w[0, 0] * y[3])
     assert np.allclose(out[1], w[1, 0] * y[0] + w[1, 1] * y[9])
     assert np.all(out[2] == 0) and np.all(out[3] == 0)                  # no local pair; dead row
+
+
+# ---------------------------------------------------------------------------------------------
+# The layer as Section 2.1 defines it (router -> dispatch -> expert FFN -> combine), written token
+# by token with no layout at all: out[t] = sum over the token's slots s, in slot order, of
+# w[t,s] * FFN_{e(t,s)}(x[t]) for the experts this rank holds.  No pair_row, no row_pair, no
+# padded buffer: it pins the token-of-pair lookup of permute_pad at k > 1, the dispatch maps and
+# the combine together, which the k = 1 dense case and the split-invariance test cannot.
+# ---------------------------------------------------------------------------------------------
+
+def _local_experts(wl):
+    """Experts with at least one replica column that the dispatch accepts (first claim of a slot wins)."""
+    claimed, local = set(), set()
+    for e in range(wl.E):
+        for r in range(wl.R_max):
+            s = int(wl.replica_map[e, r])
+            if 0 <= s < wl.G_max and s not in claimed:
+                claimed.add(s)
+                local.add(e)
+    return local
+
+
+def _per_token_definition(wl, ffn_row):
+    """ffn_row(e, x_row[1, d]) -> y[1, d] f32.  Slot order, fp32 accumulation, dead rows zero."""
+    local = _local_experts(wl)
+    out = np.zeros((wl.T, wl.d), np.float32)
+    for t in range(wl.n_valid):
+        acc = np.zeros(wl.d, np.float32)
+        for s in range(wl.k):
+            e = int(wl.topk_ids[t, s])
+            if e in local:
+                acc = acc + np.float32(wl.topk_w[t, s]) * ffn_row(e, wl.x[t:t + 1])[0]
+        out[t] = acc
+    return out
+
+
+def _fp8_ffn_row(wl):
+    def ffn_row(e, x_row):
+        w = wl.expert_weights(e)
+        q, s = O.quantise_1x128(x_row)
+        return O.expert_ffn(q, s, w.w13_q, w.w13_s, w.w2_q, w.w2_s)[2]
+    return ffn_row
+
+
+def _moe_cases():
+    stale = W.random_small(7, T=40, E=6, k=3, R_max=3, n_valid=33, stale=True)
+    return [W.config1(), W.random_small(11, T=48, E=7, k=3, R_max=3, n_valid=41), stale,
+            W.random_small(5, T=30, E=5, k=2, R_max=2)]
+
+
+@pytest.mark.parametrize("idx", range(4))
+def test_block_equals_the_per_token_moe_definition(idx):
+    wl = _moe_cases()[idx]
+    r = O.expert_block(wl)
+    ref = _per_token_definition(wl, _fp8_ffn_row(wl))
+    assert np.any(ref != 0)
+    if idx in (1, 2):
+        assert wl.n_valid < wl.T and wl.k == 3
+        assert len(_local_experts(wl)) < wl.E                      # some experts live on another rank
+        assert np.all(r["out"][wl.n_valid:] == 0)
+    assert np.array_equal(r["out"], ref)
+    # a wrong token-of-pair lookup must be visible (guards the test): shift every token by one
+    bad = np.roll(ref, 1, axis=0)
+    assert not np.array_equal(r["out"], bad)
+
+
+def test_block_equals_a_definition_that_shares_no_ffn_code():
+    """The same per-token sum with the expert written out from the definition in float64 torch ops
+    (dequantised operands, gate rows first, SwiGLU, the 1x128 quantiser in between)."""
+    wl = W.random_small(11, T=48, E=7, k=3, R_max=3, n_valid=41)
+    cache = {}
+
+    def ffn_row(e, x_row):
+        if e not in cache:
+            w = wl.expert_weights(e)
+            cache[e] = (torch.from_numpy(O.dequantise_128x128(w.w13_q, w.w13_s)),
+                        torch.from_numpy(O.dequantise_128x128(w.w2_q, w.w2_s)))
+        W13, W2 = cache[e]
+        q, s = O.quantise_1x128(x_row)
+        a = torch.from_numpy(O.dequantise_1x128(q, s))
+        gu = (a @ W13.T).float()
+        g, u = gu[:, :wl.f], gu[:, wl.f:]
+        h = (g / (1 + torch.exp(-g))) * u
+        hq, hs = O.quantise_1x128(h.numpy())
+        return (torch.from_numpy(O.dequantise_1x128(hq, hs)) @ W2.T).float().numpy()
+
+    ref = _per_token_definition(wl, ffn_row)
+    out = O.expert_block(wl)["out"]
+    scale = np.abs(ref).max()
+    assert np.abs(out - ref).max() <= 2e-3 * scale          # a rare H code may flip on exp() rounding
+    assert np.abs(out - ref).mean() <= 1e-4 * np.abs(ref).mean()
+
+
+@pytest.mark.parametrize("idx", [0, 1])
+def test_bf16_block_equals_the_per_token_moe_definition(idx):
+    wl = _moe_cases()[idx]
+
+    def ffn_row(e, x_row):
+        w13, w2 = wl.expert_weights_bf16(e)
+        return O.expert_ffn_bf16(x_row, w13, w2)[1]
+
+    r = O.expert_block_bf16(wl)
+    ref = _per_token_definition(wl, ffn_row)
+    assert np.any(ref != 0)
+    assert np.array_equal(r["out"], ref)
