@@ -11,7 +11,10 @@
  *
  * Conventions
  *   - Every pointer is a DEVICE pointer unless marked [host].  The caller owns every buffer;
- *     the library allocates nothing and keeps no state between calls.
+ *     the library allocates nothing and keeps no state between calls that a caller could observe
+ *     (two host-side caches only: the address of a driver routine, and which devices already had
+ *     a kernel's shared-memory limit raised; both are safe to fill from several threads).  The
+ *     one exception is tempo_grouped_ffn_static, which owns a device array: see there.
  *   - `stream` is a cudaStream_t passed as void*.  Every hot-path call only enqueues kernels:
  *     no host synchronisation, no host read of device data, no allocation, so the calls can be
  *     captured in a CUDA graph (the deployment the paper describes, Section 2.1 / 4.4).
@@ -73,12 +76,6 @@ enum {
 
 int tempo_version(void);
 
-/*
- * [host] Which kernel steps 3a/3b/3 use from now on in this process: 0 = the default (one CTA per
- * tile), 1 = one CTA per tile, 2 = CTA pairs.  For tests and measurements; results do not
- * depend on it.  Not thread-safe against concurrent launches.  TEMPO_ERR_SHAPE for another value.
- */
-int tempo_set_ffn_mode(int mode);
 const char* tempo_status_string(int code); /* [host] text for a TEMPO_ERR_* code */
 
 /* [host] Safe row capacity: round128(T*k) + 128*G_max (each instance pads by < 128 rows). */
@@ -131,7 +128,8 @@ int tempo_pack_weights(const tempo_shape* shape, const void* w13_q, const float*
  * columns that hold the expert, S = sum q_r (all q_r = 1 if S == 0: uniform fallback), column r
  * takes ranks [floor(C_{r-1} n_e / S), floor(C_r n_e / S)), C the running sum of q.  When
  * S == n_e every column receives exactly its share.  A pair can never go to a column whose
- * slot is -1, and nothing divides by zero.
+ * slot is -1, and nothing divides by zero.  A share above 2^30 is a malformed entry like a negative
+ * one (counts as zero, TEMPO_STATUS_BAD_TABLE), so the 64-bit products above cannot wrap.
  */
 int tempo_count_dispatch(const tempo_shape* shape, const int32_t* topk_ids, const int32_t* n_valid,
                          const int32_t* replica_map, const int32_t* quota, uint32_t* cum_counts,
@@ -164,11 +162,14 @@ int tempo_count_dispatch_sampled(const tempo_shape* shape, const int32_t* topk_i
  * integer with max|block| <= 448 * 2^eps (0 for an all-zero block), round-to-nearest-even,
  * saturating; padding rows are zero codes with scale 1.  Rows >= m_pad are not written.
  *   in   x bf16 [T, d], row_pair, m_pad        out  a_q u8 [M_cap, d], a_sf u8 [tempo_sf_bytes(M_cap, d)]
- *   pair_row (optional, may be NULL): step 1's pair -> row map.  With it, and when x is too large to
- *   stay in L2 (T*d*2 > 48 MB), the kernel walks the TOKENS, quantises each row of x once and writes it
- *   to the rows of all its local pairs, so x is read from HBM once however many local pairs a token has;
- *   otherwise it walks the rows and gathers.  Same output bit for bit.  pair_row and row_pair must come
- *   from the same step-1 call.
+ *   pair_row (optional, may be NULL): step 1's pair -> row map.  Without it the kernel walks the ROWS of
+ *   the layout and gathers.  With it the kernel may walk the TOKENS instead, quantising each row of x once
+ *   and writing it to the rows of all its local pairs: for batches small enough that every (token, 512
+ *   columns) item gets a warp of its own or up to six items per warp (decode-sized), in one wave with no
+ *   loop; and for batches whose x no longer stays in L2 between a token's gathers (T*d*2 > 48 MB), with a
+ *   grid-stride loop, so x is read from HBM once however many local pairs a token has.  In between
+ *   it walks the rows.  Same output bit for bit whichever walk runs.  pair_row and row_pair must come from
+ *   the same step-1 call.
  */
 int tempo_permute_pad(const tempo_shape* shape, const void* x_bf16, const int32_t* row_pair,
                       const int32_t* pair_row, const int32_t* m_pad, void* a_q, uint8_t* a_sf,
@@ -184,11 +185,10 @@ int tempo_permute_pad(const tempo_shape* shape, const void* x_bf16, const int32_
  * stream never pauses between the two GEMMs.  The kernel's CTAs wait for each other's H blocks
  * (bounded, one per SM): launch it on a GPU it does not have to share with another long-running
  * kernel, or the wait may time out (TEMPO_STATUS_TIMEOUT).  Rows >= m_pad are not written.
- * Two kernels implement step 3 with the same results: one CTA per 128x256 output tile (few rows per
- * instance, the flat piece of Eq. 1) and pairs of CTAs on 256x256 tiles with the weight tile split
- * between them (tcgen05 cta_group::2).  The first is the default for every shape: on B200 the pair
- * kernel measured no faster with many rows and slower with few.  Either kernel is correct for any
- * data and both give the same bits; see tempo_set_ffn_mode.
+ * Every device-side wait of the kernel gives up after 50 ms (the longest wait of a healthy launch is a
+ * few milliseconds on the largest shapes); tempo_grouped_ffn_bounded is the same call with the bound
+ * as an argument (nanoseconds, > 0), for a GPU shared through MPS or time slicing, where a CTA can be
+ * kept off its SM for longer: give it a few times the longest kernel of the co-tenant.
  */
 int tempo_ffn_gate_up(const tempo_shape* shape, const void* a_q, const uint8_t* a_sf, const void* packed,
                       const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf,
@@ -198,6 +198,10 @@ int tempo_ffn_down(const tempo_shape* shape, const void* h_q, const uint8_t* h_s
 int tempo_grouped_ffn(const tempo_shape* shape, const void* a_q, const uint8_t* a_sf, const void* packed,
                       const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y_bf16,
                       uint32_t* status, void* workspace, void* stream);
+
+int tempo_grouped_ffn_bounded(const tempo_shape* shape, const void* a_q, const uint8_t* a_sf, const void* packed,
+                              const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y_bf16,
+                              uint32_t* status, void* workspace, uint64_t wait_limit_ns, void* stream);
 
 /*
  * tempo_grouped_ffn without a caller-provided scratch buffer.  (The paper has no counterpart: this
@@ -211,8 +215,9 @@ int tempo_grouped_ffn(const tempo_shape* shape, const void* a_q, const uint8_t* 
  *   - Limit: M_cap <= 2,097,152 rows (16384 tiles of 128).  A larger M_cap returns
  *     TEMPO_ERR_UNSUPPORTED and launches nothing.
  *   - Allocates nothing, ever.  The first call on each device looks up the array's device address
- *     (cudaGetSymbolAddress, with that device current); make that first call outside any stream
- *     capture.  Every call enqueues a small cudaMemsetAsync of the counters before the kernel.
+ *     (cudaGetSymbolAddress, with that device current) and caches it on the host; make that first
+ *     call outside any stream capture, and from one thread (two threads racing on a device's first
+ *     call both look the address up and store the same value).  Every call enqueues a small cudaMemsetAsync of the counters before the kernel.
  *   - All calls on a GPU share the one array: two calls that can overlap on the GPU (different
  *     streams) race on it and give wrong results.  Serialise them, or use tempo_grouped_ffn with a
  *     buffer per stream.

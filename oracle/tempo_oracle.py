@@ -47,6 +47,9 @@ STATUS_CAPACITY = 4      # padded rows exceed M_cap: the rows that do not fit ar
 STATUS_TIMEOUT = 8       # (GPU only) a bounded device wait expired
 STATUS_BAD_SCALE = 16    # (GPU only, weight packing) a weight scale is not a power of two
 
+MAX_SHARE = 1 << 30      # a share x_{e,r} beyond this is a malformed table entry (Section 4.4: a torn or
+                         # stale row may cost a stale or uniform split, never a wrong replica)
+
 
 # ----------------------------------------------------------------------------------------
 # step 1: counts + quota dispatch + padded layout
@@ -75,7 +78,7 @@ def replica_boundaries(n_e: int, slots, quotas, G_max: int, claimed: set):
             continue
         claimed.add(s)
         valid[r] = True
-        if x < 0:
+        if x < 0 or x > MAX_SHARE:                   # malformed share: counts as zero
             status |= STATUS_BAD_TABLE
             x = 0
         q[r] = x

@@ -18,10 +18,10 @@ TEMPO_OK = 0
 STATUS_BAD_ID, STATUS_BAD_TABLE, STATUS_CAPACITY, STATUS_TIMEOUT, STATUS_BAD_SCALE = 1, 2, 4, 8, 16
 
 EXPORTS = (
-    "tempo_version", "tempo_set_ffn_mode", "tempo_status_string", "tempo_m_cap_bound", "tempo_sf_bytes", "tempo_workspace_bytes",
+    "tempo_version", "tempo_status_string", "tempo_m_cap_bound", "tempo_sf_bytes", "tempo_workspace_bytes",
     "tempo_packed_weight_bytes",
     "tempo_pack_weights", "tempo_count_dispatch", "tempo_count_dispatch_sampled", "tempo_permute_pad", "tempo_ffn_gate_up", "tempo_ffn_down",
-    "tempo_grouped_ffn", "tempo_grouped_ffn_static", "tempo_unpermute_combine",
+    "tempo_grouped_ffn", "tempo_grouped_ffn_bounded", "tempo_grouped_ffn_static", "tempo_unpermute_combine",
     "tempo_count_dispatch_masked", "tempo_permute_pad_masked", "tempo_grouped_ffn_masked",
     "tempo_packed_weight_bytes_bf16", "tempo_pack_weights_bf16", "tempo_permute_pad_bf16", "tempo_grouped_ffn_bf16",
 )
@@ -79,10 +79,6 @@ def make_shape(T, k, E, G_max, R_max, d, f, M_cap) -> TempoShape:
 
 def tempo_version() -> int:
     return _lib.tempo_version()
-
-
-def tempo_set_ffn_mode(mode: int) -> None:
-    _check(_lib.tempo_set_ffn_mode(ctypes.c_int(mode)), "tempo_set_ffn_mode")
 
 
 def tempo_m_cap_bound(shape: TempoShape) -> int:
@@ -163,6 +159,16 @@ def tempo_grouped_ffn(shape, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf
                                   _ptr(h_q, torch.uint8), _ptr(h_sf, torch.uint8), _ptr(y_bf16, torch.bfloat16),
                                   _ptr(status, torch.int32), _ptr(workspace, torch.uint8), _stream()),
            "tempo_grouped_ffn")
+
+
+def tempo_grouped_ffn_bounded(shape, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, workspace,
+                              wait_limit_ns):
+    _check(_lib.tempo_grouped_ffn_bounded(ctypes.byref(shape), _ptr(a_q, torch.uint8), _ptr(a_sf, torch.uint8),
+                                          _ptr(packed, torch.uint8), _ptr(inst_off, torch.int32),
+                                          _ptr(m_pad, torch.int32), _ptr(h_q, torch.uint8), _ptr(h_sf, torch.uint8),
+                                          _ptr(y_bf16, torch.bfloat16), _ptr(status, torch.int32),
+                                          _ptr(workspace, torch.uint8), ctypes.c_uint64(int(wait_limit_ns)), _stream()),
+           "tempo_grouped_ffn_bounded")
 
 
 def tempo_grouped_ffn_static(shape, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status):

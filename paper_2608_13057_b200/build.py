@@ -9,7 +9,7 @@ PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libtempo.so")
-SOURCES = ["api.cu", "dispatch.cu", "dispatch_sampled.cu", "permute.cu", "ffn.cu", "ffn_pair.cu", "combine.cu", "pack.cu"]
+SOURCES = ["api.cu", "dispatch.cu", "dispatch_sampled.cu", "permute.cu", "ffn.cu", "combine.cu", "pack.cu"]
 
 
 def _stale() -> bool:

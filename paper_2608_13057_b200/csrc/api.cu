@@ -27,15 +27,19 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+static EncodeTiledFn resolve_encode_fn() {
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+      q == cudaDriverEntryPointSuccess)
+    return reinterpret_cast<EncodeTiledFn>(ptr);
+  return nullptr;
+}
+
 static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;   // resolved once; a pure host-side driver routine
-  if (fn == nullptr) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
+  // A pure host-side driver routine, looked up once; the initialisation of a function-local static
+  // is thread-safe, so concurrent first calls from several threads are fine.
+  static const EncodeTiledFn fn = resolve_encode_fn();
   return fn;
 }
 
@@ -52,27 +56,6 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Flat view of a byte buffer as rows of 128 bytes, copied box_rows rows at a time, no swizzle.
-static bool make_flat_map(CUtensorMap* map, const void* base, uint64_t bytes, uint32_t box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr || bytes < 128ull * box_rows) return false;
-  const cuuint64_t dims[2] = {128, bytes / 128};
-  const cuuint64_t strides[1] = {128};
-  const cuuint32_t box[2] = {128, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// Which FFN kernel runs (tempo_set_ffn_mode): 0 = the default, 1 = one CTA per tile, 2 = CTA pairs.
-// The default is one CTA per tile for every shape: measured on B200 the pair kernel is no faster
-// with many rows per instance (both end up limited by the bytes one SM can take in per unit time,
-// and the half tile the pair's other SM supplies counts against the same limit) and slower with few.
-static int g_ffn_mode = 0;
-
-static bool use_pair_kernel(const tempo_shape*) { return g_ffn_mode == 2; }
-
 static int sm_count() {
   int dev = 0, n = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
@@ -84,7 +67,7 @@ static int sm_count() {
 static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
                            const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y,
                            uint32_t* status, void* workspace, cudaStream_t stream, int max_m = 0,
-                           const int32_t* inst_count = nullptr) {
+                           const int32_t* inst_count = nullptr, unsigned long long wait_ns = kDefaultWaitNs) {
   const PackLayout L = pack_layout(s->G_max, s->d, s->f);
   const uint8_t* blob = static_cast<const uint8_t*>(packed);
   const int sms = sm_count();
@@ -108,29 +91,14 @@ static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, 
   p.m_pad = m_pad;
   p.stride_tiles = max_m / 128;
   p.inst_count = inst_count;
-  if (max_m > 0 && use_pair_kernel(s)) return TEMPO_ERR_UNSUPPORTED;   // the pair kernel knows the grouped layout only
   p.h_q = static_cast<uint8_t*>(h_q);
   p.h_sf = h_sf;
   p.y = static_cast<__nv_bfloat16*>(y);
   p.ready = static_cast<int32_t*>(workspace);
   p.done = p.ready ? p.ready + s->M_cap / 128 : nullptr;
   p.status = status;
-  if (!use_pair_kernel(s))
-    return launch_ffn(tmA1, tmA2, tmY, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
-  PairMaps m;
-  m.a1 = tmA1; m.a2 = tmA2; m.y = tmY;
-  const size_t sf1_bytes = static_cast<size_t>(s->M_cap / 128) * L.J1 * 512, sf2_bytes = static_cast<size_t>(s->M_cap / 128) * L.J2 * 512;
-  if (!make_flat_map(&m.w, blob, L.total, 128)) return TEMPO_ERR_CUDA;
-  if (!make_flat_map(&m.sfb, blob, L.total, 8)) return TEMPO_ERR_CUDA;
-  // a side that does not run still needs a well-formed map
-  if (!make_flat_map(&m.sfa1, (run_mask & 1) ? a_sf : h_sf, (run_mask & 1) ? sf1_bytes : sf2_bytes, 4)) return TEMPO_ERR_CUDA;
-  if (!make_flat_map(&m.sfa2, h_sf, sf2_bytes, 4)) return TEMPO_ERR_CUDA;
-  PairRows pr;
-  pr.w_row[0] = static_cast<uint32_t>(L.off_w13 / 128);
-  pr.w_row[1] = static_cast<uint32_t>(L.off_w2 / 128);
-  pr.sfb_row[0] = static_cast<uint32_t>(L.off_sf13 / 128);
-  pr.sfb_row[1] = static_cast<uint32_t>(L.off_sf2 / 128);
-  return launch_ffn_pair(m, p, pr, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+  p.wait_ns = wait_ns;
+  return launch_ffn(tmA1, tmA2, tmY, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
 
 // ---- scratch for tempo_grouped_ffn_static ---------------------------------------------------------
@@ -161,12 +129,6 @@ using namespace tempo;
 extern "C" {
 
 int tempo_version(void) { return 1; }
-
-int tempo_set_ffn_mode(int mode) {
-  if (mode < 0 || mode > 2) return TEMPO_ERR_SHAPE;
-  tempo::g_ffn_mode = mode;
-  return TEMPO_OK;
-}
 
 const char* tempo_status_string(int code) {
   switch (code) {
@@ -291,6 +253,18 @@ int tempo_grouped_ffn(const tempo_shape* s, const void* a_q, const uint8_t* a_sf
                          static_cast<cudaStream_t>(stream));
 }
 
+int tempo_grouped_ffn_bounded(const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
+                              const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y_bf16,
+                              uint32_t* status, void* workspace, uint64_t wait_limit_ns, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!a_q || !a_sf || !packed || !inst_off || !m_pad || !h_q || !h_sf || !y_bf16 || !status || !workspace)
+    return TEMPO_ERR_NULL;
+  if (wait_limit_ns == 0) return TEMPO_ERR_SHAPE;
+  return launch_ffn_host(3, s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, workspace,
+                         static_cast<cudaStream_t>(stream), 0, nullptr, wait_limit_ns);
+}
+
 int tempo_grouped_ffn_static(const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
                              const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y_bf16,
                              uint32_t* status, void* stream) {
@@ -409,6 +383,7 @@ int tempo_grouped_ffn_bf16(const tempo_shape* s, const void* a_bf16, const void*
   p.ready = static_cast<int32_t*>(workspace);
   p.done = p.ready + s->M_cap / 128;
   p.status = status;
+  p.wait_ns = kDefaultWaitNs;
   return launch_ffn_bf16(tmA1, tmA2, tmY, p, sms, static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK
                                                                                                          : TEMPO_ERR_CUDA;
 }

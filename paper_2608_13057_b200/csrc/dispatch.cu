@@ -163,7 +163,9 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
       if (slot < 0 || slot >= G) continue;                       // flagged above
       if (owner[slot] != idx) { st |= TEMPO_STATUS_BAD_TABLE; continue; }
       vmask |= 1u << r;
-      if (x < 0) st |= TEMPO_STATUS_BAD_TABLE; else S += static_cast<unsigned long long>(x);
+      // a share outside [0, 2^30] is malformed and counts as zero: with at most 8 columns the running sum
+      // stays below 2^34 and C * n_e below 2^64, so the boundaries below cannot wrap
+      if (x < 0 || x > kMaxShare) st |= TEMPO_STATUS_BAD_TABLE; else S += static_cast<unsigned long long>(x);
     }
     if (cta == 0) my_status |= st;
     const bool uniform = (S == 0);
@@ -174,7 +176,8 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
     for (int r = 0; r < R; ++r) {
       const int idx = e * R + r;
       const bool valid = (vmask >> r) & 1u;
-      if (valid) C += uniform ? 1ull : static_cast<unsigned long long>(max(quota_s[idx], 0));
+      const int xq = quota_s[idx];
+      if (valid) C += uniform ? 1ull : static_cast<unsigned long long>((xq < 0 || xq > kMaxShare) ? 0 : xq);
       int B = 0;
       if (S > 0) {
         if (C < 65536ull && S < 65536ull && n_e < 65536)

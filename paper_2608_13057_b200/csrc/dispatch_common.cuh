@@ -9,7 +9,9 @@ constexpr int kDispThreads = 1024;
 constexpr int kDispWarps = kDispThreads / 32;
 constexpr int kKeep = 4;           // 32-pair steps of a warp whose ids stay in registers between the passes
 constexpr int kMaxCluster = 8;     // portable cluster size
-constexpr int kPairsPerCta = 1024; // pairs per CTA before another CTA joins the cluster
+constexpr int kPairsPerCta = 1024;
+constexpr int kMaxShare = 1 << 30;   // largest share x_{e,r} the quota dispatch accepts
+constexpr size_t kDispatchSmemLimit = 220 * 1024;   // the shape check rejects tables beyond this // pairs per CTA before another CTA joins the cluster
 
 // Lanes of the warp that hold the same expert id as this lane (e < 0: none).  One ballot per id
 // bit: a fixed, short latency, where __match_any_sync takes one round per distinct value.
@@ -63,7 +65,9 @@ inline int dispatch_cluster_size(long long pairs) {
 template <typename Params>
 inline cudaError_t launch_dispatch_cluster(void (*kernel)(Params), const Params& p, long long pairs, size_t smem,
                                            cudaStream_t stream) {
-  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  // (the limit is raised to the largest table the shape checks admit, once per device and kernel)
+  static std::atomic<unsigned long long> smem_set{0};
+  cudaError_t e = smem_limit_once(kernel, kDispatchSmemLimit, smem_set);
   if (e != cudaSuccess) return e;
   const int nc = dispatch_cluster_size(pairs);
   cudaLaunchConfig_t cfg = {};

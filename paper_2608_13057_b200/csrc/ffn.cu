@@ -32,7 +32,7 @@
 // Scales are UE8M0 per 128 K-elements; the MMA takes one scale byte per row (A) and per column
 // (B) for each K=32 step, so the four steps of a K-block select the same byte (scale id kb % 4).
 //
-// Every wait is bounded: after kWaitLimitNs the CTA raises an abort flag, all roles leave their
+// Every wait is bounded: after FfnParams::wait_ns the CTA raises an abort flag, all roles leave their
 // loops, TEMPO_STATUS_TIMEOUT is set and tensor memory is freed.
 #include "ffn_common.cuh"
 
@@ -69,6 +69,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const int G = p.G_max;
+  const unsigned long long wait_ns = p.wait_ns;
   pdl_trigger();
   // prologue that needs nothing from the previous kernel: barriers, tensor memory, descriptor fetch
   if (tid == 0) {
@@ -157,7 +158,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         const bool stream_b = w.m_tiles <= 2;
 #pragma unroll 1
         for (int kb = 0; kb < gs.Kb; ++kb) {
-          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
           const uint32_t full = smem_u32(&s_full[stage]);
           const uint32_t sB = smem_base + stage * kStageBytes + kABytes, sSF = sB + kBBytes;
           const bool with_sf = !kBf16 && (kb & 3) == 0;
@@ -191,7 +192,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
               if (*s_abort) { ok = false; break; }
               const unsigned long long now = global_timer_ns();
               if (t0 == 0) t0 = now;
-              else if (now - t0 > kWaitLimitNs) { *s_abort = 1; ok = false; break; }
+              else if (now - t0 > wait_ns) { *s_abort = 1; ok = false; break; }
             }
           }
           if (!ok) break;
@@ -203,7 +204,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
         }
 #pragma unroll 1
         for (int kb = 0; kb < gs.Kb; ++kb) {
-          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
           const uint32_t full = smem_u32(&s_full[stage]);
           const uint32_t sA = smem_base + stage * kStageBytes, sSF = sA + kABytes + kBBytes;
           const bool with_sf = !kBf16 && (kb & 3) == 0;
@@ -235,7 +236,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
             if (*s_abort) { ok = false; break; }
             const unsigned long long now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) { *s_abort = 1; ok = false; break; }
+            else if (now - t0 > wait_ns) { *s_abort = 1; ok = false; break; }
           }
         }
         if (!ok) break;
@@ -256,11 +257,11 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       int side, x;
       while (ok && it.next(side, x)) {
         const int Kb = p.side[side].Kb;
-        if (!mbar_wait(smem_u32(&s_acc_empty), acc_phase ^ 1u, s_abort)) break;
+        if (!mbar_wait(smem_u32(&s_acc_empty), acc_phase ^ 1u, s_abort, wait_ns)) break;
         tc_fence_after();
 #pragma unroll 1
         for (int kb = 0; kb < Kb; ++kb) {
-          if (!mbar_wait(smem_u32(&s_full[stage]), phase, s_abort)) { ok = false; break; }
+          if (!mbar_wait(smem_u32(&s_full[stage]), phase, s_abort, wait_ns)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sA = smem_base + stage * kStageBytes, sB = sA + kABytes, sSF = sB + kBBytes;
           const uint32_t sfa_t = tmem_base + kSfCol0 + 16u * ((kb >> 2) & 1);
@@ -313,7 +314,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
       const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2, stride);
       const int row = w.row0 + r_in_tile;
       // Both warps of a pair must take the same way out: they vote on the outcome of the wait.
-      const bool ok = mbar_wait(smem_u32(&s_acc_full), acc_phase, s_abort);
+      const bool ok = mbar_wait(smem_u32(&s_acc_full), acc_phase, s_abort, wait_ns);
       acc_phase ^= 1u;
       if (lane == 0) s_ok[par][quad][half] = ok ? 1 : 0;
       pair_sync(pair_bar);
@@ -489,8 +490,8 @@ size_t ffn_workspace_bytes(int M_cap) {
 template <bool kBf16>
 static cudaError_t launch_ffn_t(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
                                 const FfnParams& p, int num_sms, cudaStream_t stream) {
-  cudaError_t e = cudaFuncSetAttribute(ffn_kernel<kBf16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(kGemmSmemBytes));
+  static std::atomic<unsigned long long> smem_set{0};
+  cudaError_t e = smem_limit_once(ffn_kernel<kBf16>, kGemmSmemBytes, smem_set);
   if (e != cudaSuccess) return e;
   const int grid = max(1, num_sms);   // one persistent CTA per SM; CTAs without work leave at once
   return launch_pdl(ffn_kernel<kBf16>, dim3(grid), dim3(kGemmThreads), kGemmSmemBytes, stream, tmA1, tmA2, tmY, p);

@@ -1,6 +1,6 @@
-// Pieces shared by the two fused FFN kernels (one CTA per tile, and CTA pairs): tile geometry,
-// PTX wrappers for mbarriers, bulk/tensor copies and the tcgen05 instructions, shared-memory and
-// instruction descriptors, and the static tile assignment.
+// Building blocks of the fused FFN kernel: tile geometry, PTX wrappers for mbarriers, bulk/tensor
+// copies and the tcgen05 instructions, shared-memory and instruction descriptors, and the static
+// tile assignment.
 #pragma once
 
 #include <cuda.h>
@@ -19,7 +19,6 @@ constexpr int kTileOverhead = 5;                          // per-tile fixed cost
 constexpr int kTmemCols = 512;
 constexpr int kSfCol0 = 256;                              // scale slot s: A at 256+16s, B at 260+16s
 constexpr int kMaxSlots = 1024;
-constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 constexpr int kStoreBytes = 32 * 128;                       // per-warp staging of a TMA store: 32 rows x 128 bytes
 
 
@@ -46,8 +45,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out of time).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait (limit in ns).  Returns false if the CTA is aborting (this wait or another one ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns) {
   unsigned long long t0 = 0;
   for (uint32_t it = 0;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -55,7 +55,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const unsigned long long now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
   }
 }

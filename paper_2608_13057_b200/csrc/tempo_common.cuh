@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "tempo.h"
 
 namespace tempo {
@@ -60,6 +62,24 @@ __device__ __forceinline__ uint32_t cvt_e4m3x4(float a, float b, float c, float 
 // kernel's tail.  Both are no-ops when the kernel was launched without the attribute.
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Default bound of the device-side waits of the FFN kernel (tempo_grouped_ffn_bounded takes another).
+constexpr unsigned long long kDefaultWaitNs = 50ull * 1000ull * 1000ull;
+
+// Raises a kernel's dynamic shared-memory limit once per device and kernel instead of on every launch.
+// `done` is a bit mask over device ordinals owned by the caller (one static per kernel); a race between
+// two first calls sets the attribute twice, which is harmless.
+template <typename Kernel>
+inline cudaError_t smem_limit_once(Kernel kernel, size_t bytes, std::atomic<unsigned long long>& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = dev >= 0 && dev < 64 ? 1ull << dev : 0ull;
+  if (bit != 0 && (done.load(std::memory_order_acquire) & bit)) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+  if (e == cudaSuccess && bit != 0) done.fetch_or(bit, std::memory_order_release);
+  return e;
+}
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,

@@ -111,6 +111,7 @@ struct FfnParams {
   int32_t* ready;        // workspace: per M-tile, epilogue warps of finished gate/up tiles
   int32_t* done;         // workspace: per M-tile, down tiles that have seen `ready` complete
   uint32_t* status;
+  unsigned long long wait_ns;   // bound of every device-side wait of the kernel, in nanoseconds
 };
 size_t ffn_workspace_bytes(int M_cap);
 // The bf16 variant: Kb counts 64-value K-blocks, the scale pointers and J_h are unused, h_q holds bf16.
@@ -119,20 +120,5 @@ cudaError_t launch_ffn_bf16(const CUtensorMap& tmA1, const CUtensorMap& tmA2, co
 cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
                        const FfnParams& p, int num_sms, cudaStream_t stream);
 
-
-// The CTA-pair kernel for many rows per instance (ffn_pair.cu).  It reads the packed weights and
-// the scale buffers through flat views (rows of 128 bytes); PairRows says where the sections of
-// the packed blob start in that view.
-struct PairRows {
-  uint32_t w_row[2];     // packed B tiles of side 0 / 1: 256 rows per (instance, tile, K-block)
-  uint32_t sfb_row[2];   // scale atoms of the packed weights: 8 rows per (instance, tile, j)
-};
-struct PairMaps {
-  CUtensorMap a1, a2;    // activations of the two GEMMs, 128-row boxes, 128-byte swizzle
-  CUtensorMap y;         // Y stores, 32-row boxes
-  CUtensorMap w, sfb;    // flat views of the packed blob: 128-row and 8-row boxes
-  CUtensorMap sfa1, sfa2;  // flat views of the activation scale buffers: 4-row boxes
-};
-cudaError_t launch_ffn_pair(const PairMaps& m, const FfnParams& p, const PairRows& pr, int num_sms, cudaStream_t stream);
 
 }  // namespace tempo

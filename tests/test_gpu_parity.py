@@ -84,6 +84,11 @@ def _dispatch_cases():
     yield _table_case(np.zeros((40, 1)), 40, [[0, 9, 1]], [[20, 10, 20]], 4, "slot-out-of-range")
     yield _table_case(np.zeros((40, 1)), 40, [[0, 1, -1]], [[-5, 40, 0]], 4, "negative-share")
     yield _table_case([[0], [1], [1], [0]], 4, [[0], [0]], [[2], [2]], 1, "slot-claimed-twice")
+    # absurd shares (torn table): beyond 2^30 an entry counts as zero, so the split can never wrap
+    big = 2 ** 31 - 1
+    yield _table_case(np.zeros((300, 1)), 300, [[0, 1, 2]], [[big, big, 7]], 3, "huge-shares")
+    yield _table_case(np.zeros((300, 1)), 300, [[0, 1, 2]], [[big, big, big]], 3, "all-huge-shares")
+    yield _table_case(np.zeros((300, 1)), 300, [[0, 1, 2]], [[2 ** 30, 2 ** 30, 2 ** 29]], 3, "largest-legal-shares")
     yield _table_case([[0], [5], [-1], [0]], 4, [[0]], [[2]], 1, "bad-ids")
     # an expert with n_e = 0 but a non-zero share; duplicate expert inside one token; E not a multiple of 32
     ids = g.integers(1, 37, size=(64, 4))
@@ -283,6 +288,59 @@ def _sampled_rows_check(B, wl, buf, rows_per_inst=6, n_tokens=48, seed=0):
     mx, mean = _err(out_gpu, out_ref)
     assert mx <= MAX_TOL and mean <= MEAN_TOL, ("out rows", mx, mean)
     assert not (int(buf.status.item()) & B.STATUS_TIMEOUT)
+
+
+def _full_instance_check(wl, buf, ref, i):
+    """Every padded row of instance slot i (all its M-tiles, the true d and f) against the oracle: the
+    quantised activations bytewise, H through its dequantised values, Y within the FFN tolerance."""
+    lo, hi = int(ref["inst_off"][i]), int(ref["inst_off"][i + 1])
+    m = int(ref["inst_count"][i])
+    assert hi > lo and m > 0
+    rp = ref["row_pair"][lo:hi]
+    assert np.all(rp[:m] >= 0) and np.all(rp[m:] < 0)
+    a_q = np.zeros((hi - lo, wl.d), np.uint8)
+    a_s = np.ones((hi - lo, wl.d // 128), np.float32)
+    a_q[:m], a_s[:m] = O.quantise_1x128(wl.x[rp[:m] // wl.k])
+    assert codes_equal_mod_signed_zero(to_np(buf.a_q[lo:hi]), a_q).all()
+    assert np.array_equal(sf_decode(to_np(buf.a_sf), buf.M_cap, buf.d)[lo:hi], a_s)
+    w = wl.expert_weights(int(wl.slot_expert[i]))
+    h_q, h_s, y_ref = O.expert_ffn(a_q, a_s, w.w13_q, w.w13_s, w.w2_q, w.w2_s)
+    h_gpu = O.dequantise_1x128(to_np(buf.h_q[lo:hi]), sf_decode(to_np(buf.h_sf), buf.M_cap, buf.f)[lo:hi])
+    mx, mean = _err(h_gpu, O.dequantise_1x128(h_q, h_s))
+    assert mx <= 0.07 and mean <= MEAN_TOL, ("H", i, mx, mean)
+    mx, mean = _err(to_np(buf.y[lo:hi]), y_ref)
+    assert mx <= MAX_TOL and mean <= MEAN_TOL, ("Y", i, mx, mean)
+    assert np.all(to_np(buf.y[lo + m:hi]) == 0)                      # padding rows give exact zeros
+    return (hi - lo) // 128
+
+
+def test_mixed_config_hot_instance_in_full(B):
+    """Config 3 at its true shape (d=4096, f=1536): the hottest instance of the keep-hot-whole split
+    (about 30 M-tiles, dealt as a hot instance beside cold ones) compared row by row, not sampled."""
+    wl = W.config3("hot_whole")
+    buf = _run_block(B, wl)
+    ref = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    hot = int(np.argmax(ref["inst_count"]))
+    tiles = _full_instance_check(wl, buf, ref, hot)
+    assert tiles >= 24
+    cold = int(np.argmin(np.where(ref["inst_count"] > 0, ref["inst_count"], 1 << 30)))
+    _full_instance_check(wl, buf, ref, cold)
+    assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
+
+
+def test_prefill_config_multi_tile_instance_in_full(B):
+    """Config 4 at its true shape (d=7168, f=2048): one instance of several M-tiles row by row."""
+    wl = W.config4()
+    buf = _run_block(B, wl)
+    ref = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, buf.M_cap)
+    _assert_dispatch_equal(dispatch_outputs(buf), ref)
+    cnt = ref["inst_count"].astype(np.int64)
+    multi = [i for i in range(wl.G_max) if 4 * 128 < cnt[i] <= 12 * 128]     # 5 to 12 tiles: seconds on the host
+    assert multi, cnt
+    i = multi[len(multi) // 2]
+    assert _full_instance_check(wl, buf, ref, i) >= 5
+    assert int(buf.status.item()) == 0 and int(buf.workspace.max().item()) == 0
 
 
 def test_mixed_config_three_splits_sampled_and_split_invariant(B):
@@ -525,7 +583,7 @@ def test_consecutive_steps_with_different_inputs_do_not_mix(B):
 
 def test_bounded_wait_reports_timeout_and_the_context_stays_usable(B):
     """Failure detection without a fault: the down tiles wait for H-ready counters that nothing will
-    complete (the workspace is poisoned on the host), the wait gives up after its one-second limit,
+    complete (the workspace is poisoned on the host), the wait gives up after its limit (20 ms here),
     the kernel sets TEMPO_STATUS_TIMEOUT and returns; after re-zeroing the workspace the same buffers
     produce the right result again."""
     wl = W.config1()
@@ -533,9 +591,9 @@ def test_bounded_wait_reports_timeout_and_the_context_stays_usable(B):
     good = buf.y.clone()
     buf.workspace.view(torch.int32).fill_(-1000000)        # counters can never reach their target
     buf.status.zero_()
-    B.tempo_grouped_ffn(buf.shape, buf.a_q, buf.a_sf, buf.packed, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
-                        buf.status, buf.workspace)
-    torch.cuda.synchronize()                                # returns after about one second
+    B.tempo_grouped_ffn_bounded(buf.shape, buf.a_q, buf.a_sf, buf.packed, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf,
+                                buf.y, buf.status, buf.workspace, 20_000_000)
+    torch.cuda.synchronize()                                # returns after about 20 ms
     assert int(buf.status.item()) & B.STATUS_TIMEOUT
     buf.workspace.zero_()
     buf.status.zero_()

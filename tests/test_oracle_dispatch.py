@@ -195,6 +195,19 @@ def test_bad_entries_are_flagged_and_ignored():
     assert r["counts"].tolist() == [2] and r["pair_row"].tolist() == [0, -1, -1, 1]
 
 
+def test_absurd_shares_count_as_zero_and_never_pick_a_wrong_replica():
+    big = 2 ** 31 - 1
+    r = _one_expert(300, [0, 1, 2], [big, big, 7])      # two torn entries: the third column takes everything
+    assert int(r["status"]) & O.STATUS_BAD_TABLE
+    assert r["inst_count"][:3].tolist() == [0, 0, 300]
+    r = _one_expert(300, [0, 1, 2], [big, big, big])    # nothing usable left: uniform over the holders
+    assert int(r["status"]) & O.STATUS_BAD_TABLE
+    assert r["inst_count"][:3].tolist() == [100, 100, 100]
+    r = _one_expert(300, [0, 1, 2], [2 ** 30, 2 ** 30, 2 ** 29])   # the largest legal shares, 2:2:1
+    assert int(r["status"]) == 0
+    assert r["inst_count"][:3].tolist() == [120, 120, 60]
+
+
 def test_padding_rows_are_masked_and_counter_wraps():
     wl = W.config2(n_valid=200)
     cum = np.full(wl.E, 2 ** 32 - 3, np.uint32)
