@@ -1,13 +1,16 @@
 #!/usr/bin/env python
 """Benchmark of the per-rank MoE expert block on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3-uniform|...] [--impl reference]
-    python bench.py --sweep            # cost-profile sweep (G, N grid) + max-affine fit -> n*
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg3-uniform|cfg4|...] [--impl reference]
+    python bench.py --sweep            # full cost-profile sweep (G, N grid) + max-affine fit -> n*
 
-One "step" is one pass of the whole hot path (count+dispatch, permute+quantise, the fused gate/up + SwiGLU +
-down FFN kernel, combine) over one seeded synthetic routed batch, replayed as one CUDA graph.  Weight copies
-rotate through a pool larger than L2 so no step finds its weights cached (the paper's calibration
-protocol, Appendix B).  Rank 0 prints ONE JSON line.
+One "step" is one pass of the whole hot path (count+dispatch, activation quantise/permute, the fused gate/up +
+SwiGLU + down FFN kernel, combine) over one seeded synthetic routed batch, replayed from CUDA graphs.  Weight
+copies rotate through a pool larger than L2 so no step finds its weights cached (the paper's calibration
+protocol, Appendix B).  Rank 0 prints ONE JSON line.  The default line is quoted on config 2 (the flat,
+HBM-bound regime) and, at one GPU, carries the rest of the metric as well: `regimes.linear` (config 4, the
+tensor-bound regime), `fit` (Eq. 1 / Eq. 3 fitted to a reduced in-run sweep, with the B200 n*), and a dense fp8
+GEMM rate measured in the same run as the tensor-bound denominator.
 """
 from __future__ import annotations
 
@@ -15,6 +18,7 @@ import argparse
 import json
 import math
 import os
+import re
 import subprocess
 import sys
 import tempfile
@@ -30,13 +34,29 @@ METRIC = "moe_expert_block_us"          # step time / activated expert instances
 UNIT = "us_per_expert_block"
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_FP8_OVER_BF16 = 2.0             # dense fp8 peak = 2 x dense bf16 peak on this part
+NOMINAL_FP8_TFLOPS = 4500.0
+POOL_BYTES = 1 << 30                    # weight copies rotate through at least this much (>> L2)
+FIT_G = (4, 16, 64)                     # reduced in-run sweep behind `fit` (the full grid: --sweep)
+FIT_N = (64, 128, 129, 256, 1024, 4096)
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused FFN kernel from the committed ncu
-# capture (profiles/), keyed by workload; None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {
-    "cfg2": 395.02e6,          # profiles/ffn_kernel_cfg2_flat_decode.md (391.08 MB read + 3.9 MB written)
-    "cfg5-8-1024": 231.6e6,    # profiles/ffn_kernel_cfg5_G8_N1024_linear.md
+# ncu summary (profiles/) that holds dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant
+# kernel for a workload, on a line "dram_bytes_per_launch: <number>"; None where no capture exists.
+NCU_SUMMARY = {
+    "cfg2": "ffn_kernel_cfg2_flat_decode.md",
+    "cfg5-8-1024": "ffn_kernel_cfg5_G8_N1024_linear.md",
 }
+
+
+def ncu_traffic_bytes(workload: str):
+    name = NCU_SUMMARY.get(workload)
+    if name is None:
+        return None
+    try:
+        text = open(os.path.join(ROOT, "profiles", name)).read()
+    except OSError:
+        return None
+    m = re.search(r"dram_bytes_per_launch:\s*([0-9.eE+]+)", text)
+    return float(m.group(1)) if m else None
 
 
 def _peaks():
@@ -85,6 +105,20 @@ def workload_stats(wl):
                 n_valid=int(wl.n_valid), counts_total=int(counts.sum()))
 
 
+def n_pools_for(weight_bytes_all: int) -> int:
+    return min(64, max(2, math.ceil(POOL_BYTES / max(weight_bytes_all, 1))))
+
+
+def workload_config(name, wl, st, world, max_m=0):
+    """The `config` object of the JSON line: the workload and how L2 is defeated.  Both arms print the same."""
+    packed_bytes = wl.G_max * 3 * wl.d * wl.f            # + 0.8 % scale atoms
+    pools = n_pools_for(packed_bytes)
+    return {"workload": name, "T": wl.T, "top_k": wl.k, "E": wl.E, "d": wl.d, "f": wl.f, "G_act": st["G_act"],
+            "N_local": st["N_local"], "M_pad": st["M_pad"], "layout": f"masked, max_m={max_m}" if max_m else "grouped",
+            "l2": f"weights rotate through {pools} copies of {packed_bytes / 1e9:.2f} GB each (>> 126 MB L2)",
+            "parallelism": f"{world} independent rank(s), no collective"}
+
+
 class ClockSampler:
     """nvidia-smi clocks / throttle reasons sampled in the background while the GPU is timed."""
 
@@ -110,7 +144,7 @@ class ClockSampler:
                 self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         for line in self.file:
             c = [v.strip() for v in line.split(",")]
             if len(c) < 9:
@@ -118,6 +152,7 @@ class ClockSampler:
             try:
                 sm.append(float(c[1]))
                 mx.append(float(c[2]))
+                pw.append(float(c[3]))
             except ValueError:
                 continue
             for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
@@ -128,7 +163,8 @@ class ClockSampler:
         if not sm:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
         busy = [v for v in sm if v >= 0.5 * max(sm)] or sm
-        return dict(sm_mhz=float(np.median(busy)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return dict(sm_mhz=float(np.median(busy)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm),
+                    power_w_max=float(max(pw)) if pw else None)
 
 
 # --------------------------------------------------------------------------------------------------
@@ -185,7 +221,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": len(vals),
         "warmup": min(args.warmup, 1), "ms_per_step": v * st["G_act"] / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "G_act": st["G_act"], "N_local": st["N_local"]},
+        "config": workload_config(args.workload, wl, st, max(1, args.gpus), args.max_m),
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -195,8 +231,11 @@ def run_reference(args):
 # GPU arm
 # --------------------------------------------------------------------------------------------------
 
-def _capture_graphs(torch, buf, pools, run=None):
-    run = buf.run_block if run is None else run
+def _pct(ts):
+    return dict(p10=float(np.percentile(ts, 10)), p50=float(np.percentile(ts, 50)), p90=float(np.percentile(ts, 90)))
+
+
+def _capture_graphs(torch, pools, run):
     graphs = []
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
@@ -213,10 +252,9 @@ def _capture_graphs(torch, buf, pools, run=None):
     return graphs
 
 
-def _capture_chain(torch, buf, pools, steps, run=None):
+def _capture_chain(torch, pools, steps, run):
     """One graph holding `steps` consecutive steps (weight copies in rotation), as a serving stack captures
     a whole forward pass: step i+1's first kernel launches programmatically behind step i's last one."""
-    run = buf.run_block if run is None else run
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
         for i in range(steps):
@@ -224,136 +262,195 @@ def _capture_chain(torch, buf, pools, steps, run=None):
     return g
 
 
-def run_gpu(args):
-    import torch
-    import torch.distributed as dist
-    from paper_2608_13057_b200 import binding as B
-    from paper_2608_13057_b200.ranks import reduce_step
+def measure_fp8_peak(torch, seconds: float = 3.0):
+    """Dense e4m3 GEMM rate of the vendor library (torch._scaled_mm, 8192^3, per-tensor scales, bf16 out):
+    best of 10 launches (burst) and a back-to-back loop of about `seconds` (sustained, under the power cap).
+    A denominator for the tensor-bound roofline only; nothing on the hot path calls it."""
+    try:
+        n = 8192
+        a = (torch.randn(n, n, device="cuda") * 0.5).to(torch.float8_e4m3fn)
+        b = (torch.randn(n, n, device="cuda") * 0.5).to(torch.float8_e4m3fn).t()      # column-major operand
+        one = torch.ones((), device="cuda", dtype=torch.float32)
 
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        def mm():
+            return torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
 
-    wl = make_workload(args.workload, rank)
-    st = workload_stats(wl)
-    max_m = args.max_m                                 # > 0: the masked layout, instance i at rows [i*max_m, (i+1)*max_m)
-    buf = B.RankBuffers.for_workload(wl, M_cap=wl.G_max * max_m if max_m else None)
-    weight_bytes_all = buf.packed.numel()
-    n_pools = max(2, math.ceil((1 << 30) / max(weight_bytes_all, 1)))
-    n_pools = min(n_pools, 64)
-    pools = [buf.packed] + [buf.packed.clone() for _ in range(n_pools - 1)]
-    run_fn = (lambda packed: buf.run_block_masked(max_m, packed=packed)) if max_m else None
-    graphs = _capture_graphs(torch, buf, pools, run_fn)
-    K, Wm = args.steps, args.warmup
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
+        for _ in range(3):
+            mm()
         torch.cuda.synchronize()
+        flops = 2.0 * n ** 3
+        best = float("inf")
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            mm()
+            e1.record()
+            e1.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        reps = max(10, int(seconds * 1e3 / best))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            mm()
+        e1.record()
+        e1.synchronize()
+        sustained = e0.elapsed_time(e1) / reps
+        return dict(fp8_tflops=flops / best / 1e9, fp8_tflops_sustained=flops / sustained / 1e9,
+                    how=f"torch._scaled_mm e4m3 x e4m3 -> bf16, {n}^3, best of 10 and {reps} back to back "
+                        f"({e0.elapsed_time(e1) / 1e3:.1f} s)")
+    except Exception as exc:                             # no fp8 GEMM in this torch build: fall back to 2 x bf16
+        return dict(fp8_tflops=None, fp8_tflops_sustained=None, how=f"unavailable: {type(exc).__name__}: {exc}"[:200])
 
-    sampler = ClockSampler(local) if rank == 0 else None
 
-    # ---- region A: the whole block as one graph replay per step, inputs resident in HBM ------------
-    for i in range(Wm):
-        graphs[i % n_pools].replay()
-    barrier()
-    # K steps exactly: whole chains of `chain_steps` steps, then single-step graphs for the remainder
-    chain_steps = n_pools * max(1, 12 // n_pools)
-    chain = _capture_chain(torch, buf, pools, chain_steps, run_fn) if K >= chain_steps else None
-    if chain is not None:
-        chain.replay()
-        barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    done = 0
-    while chain is not None and K - done >= chain_steps:
-        chain.replay()
-        done += chain_steps
-    for i in range(K - done):
-        graphs[i % n_pools].replay()
-    e1.record()
-    barrier()
-    ms_total = e0.elapsed_time(e1)
-    status = int(buf.status.item())
+def tensor_denominators(peaks, fp8):
+    """TFLOP/s figures a tensor-bound fraction can be quoted against; the first available one is primary."""
+    d = {}
+    if fp8 and fp8.get("fp8_tflops_sustained"):
+        d["fp8_measured_sustained"] = fp8["fp8_tflops_sustained"]
+        d["fp8_measured_burst"] = fp8["fp8_tflops"]
+    d["bf16_sustained_x2"] = peaks["bf16_tflops_sustained"] * NOMINAL_FP8_OVER_BF16
+    d["bf16_burst_x2"] = peaks["bf16_tflops"] * NOMINAL_FP8_OVER_BF16
+    d["nominal_dense_fp8"] = NOMINAL_FP8_TFLOPS
+    return d
 
-    # ---- region B: the same steps launched call by call with events between the kernels -----------
-    Kb = min(K, 200)
-    names = ["count_dispatch", "permute_pad", "grouped_ffn", "unpermute_combine"]
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(Kb)]
-    s = buf.shape
-    torch.cuda._sleep(int(4e7))                        # keep the GPU busy so every launch is queued ahead
-    for i in range(Kb):
-        blob = pools[i % n_pools]
-        ev[i][0].record()
-        if max_m:
-            B.tempo_count_dispatch_masked(s, max_m, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts,
-                                          buf.counts, buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair,
-                                          buf.tile_inst, buf.m_pad, buf.status)
-            ev[i][1].record()
-            B.tempo_permute_pad_masked(s, buf.x, buf.row_pair, buf.pair_row, buf.tile_inst, buf.m_pad, buf.a_q, buf.a_sf,
-                                       buf.status)
-            ev[i][2].record()
-            B.tempo_grouped_ffn_masked(s, max_m, buf.a_q, buf.a_sf, blob, buf.inst_count, buf.h_q, buf.h_sf, buf.y,
-                                       buf.status, buf.workspace)
+
+class Leg:
+    """One workload on the device: buffers, weight copies, graphs, and the timed regions."""
+
+    def __init__(self, torch, B, name, wl, max_m=0, device_weights=False):
+        from paper_2608_13057_b200 import workloads as W
+        self.torch, self.B, self.name, self.wl, self.max_m = torch, B, name, wl, max_m
+        self.st = workload_stats(wl)
+        M_cap = wl.G_max * max_m if max_m else None
+        if device_weights:
+            self.buf = B.RankBuffers.for_workload(wl, M_cap=M_cap, with_weights=False)
+            self.buf.pack_weights(*W.slot_weights_cuda(wl))
+            torch.cuda.empty_cache()
         else:
-            B.tempo_count_dispatch(s, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts, buf.counts,
-                                   buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair, buf.tile_inst, buf.m_pad,
-                                   buf.status)
-            ev[i][1].record()
-            B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status, pair_row=buf.pair_row)
-            ev[i][2].record()
-            B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
-                                buf.status, buf.workspace)
-        ev[i][3].record()
-        B.tempo_unpermute_combine(s, buf.y, buf.pair_row, buf.topk_w, buf.n_valid, buf.out, buf.status)
-        ev[i][4].record()
-    torch.cuda.synchronize()
-    kern_us = {n: float(np.mean([ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(Kb)])) * 1e3
-               for j, n in enumerate(names)}
+            self.buf = B.RankBuffers.for_workload(wl, M_cap=M_cap)
+        buf = self.buf
+        self.n_pools = n_pools_for(buf.packed.numel())
+        self.pools = [buf.packed] + [buf.packed.clone() for _ in range(self.n_pools - 1)]
+        self.run = (lambda packed: buf.run_block_masked(max_m, packed=packed)) if max_m else buf.run_block
+        self.graphs = _capture_graphs(torch, self.pools, self.run)
+        self.chain_steps = self.n_pools * max(1, 12 // self.n_pools)
+        self.chain = None
 
-    # ---- e2e: host buffers in, host result out, every step ------------------------------------------
+    def replay_steps(self, K):
+        """Exactly K steps: whole chains of `chain_steps` steps, then single-step graphs for the remainder."""
+        done = 0
+        while self.chain is not None and K - done >= self.chain_steps:
+            self.chain.replay()
+            done += self.chain_steps
+        for i in range(K - done):
+            self.graphs[i % self.n_pools].replay()
+
+    def time_regions(self, K, warmup, regions, barrier):
+        torch = self.torch
+        for i in range(warmup):
+            self.graphs[i % self.n_pools].replay()
+        barrier()
+        if K >= self.chain_steps and self.chain is None:
+            self.chain = _capture_chain(torch, self.pools, self.chain_steps, self.run)
+            self.chain.replay()
+            barrier()
+        ms = []
+        for _ in range(regions):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            barrier()
+            e0.record()
+            self.replay_steps(K)
+            e1.record()
+            barrier()
+            ms.append(e0.elapsed_time(e1))
+        return ms
+
+    def kernel_pass(self, Kb):
+        """The same steps launched call by call with events between the kernels (queued behind a spin kernel so
+        that no launch is late): per-kernel CUDA-event durations on the launching stream."""
+        torch, B, buf, max_m = self.torch, self.B, self.buf, self.max_m
+        names = ["count_dispatch", "permute_pad", "grouped_ffn", "unpermute_combine"]
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(Kb)]
+        s = buf.shape
+        torch.cuda._sleep(int(4e7))
+        for i in range(Kb):
+            blob = self.pools[i % self.n_pools]
+            ev[i][0].record()
+            if max_m:
+                B.tempo_count_dispatch_masked(s, max_m, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota,
+                                              buf.cum_counts, buf.counts, buf.inst_count, buf.inst_off, buf.pair_row,
+                                              buf.row_pair, buf.tile_inst, buf.m_pad, buf.status)
+                ev[i][1].record()
+                B.tempo_permute_pad_masked(s, buf.x, buf.row_pair, buf.pair_row, buf.tile_inst, buf.m_pad, buf.a_q,
+                                           buf.a_sf, buf.status)
+                ev[i][2].record()
+                B.tempo_grouped_ffn_masked(s, max_m, buf.a_q, buf.a_sf, blob, buf.inst_count, buf.h_q, buf.h_sf, buf.y,
+                                           buf.status, buf.workspace)
+            else:
+                B.tempo_count_dispatch(s, buf.topk_ids, buf.n_valid, buf.replica_map, buf.quota, buf.cum_counts,
+                                       buf.counts, buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair,
+                                       buf.tile_inst, buf.m_pad, buf.status)
+                ev[i][1].record()
+                B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status,
+                                    pair_row=buf.pair_row)
+                ev[i][2].record()
+                B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
+                                    buf.status, buf.workspace)
+            ev[i][3].record()
+            B.tempo_unpermute_combine(s, buf.y, buf.pair_row, buf.topk_w, buf.n_valid, buf.out, buf.status)
+            ev[i][4].record()
+        torch.cuda.synchronize()
+        return {n: float(np.median([ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(Kb)])) * 1e3
+                for j, n in enumerate(names)}
+
+    def rooflines(self, us_step, kern_us, peaks, fp8):
+        """`roofline` (the dominant kernel) and `block_roofline` (the whole step) of this leg."""
+        st = self.st
+        denoms = tensor_denominators(peaks, fp8)
+        primary = next(iter(denoms))
+        fp8_peak = denoms[primary]
+        hbm_time = st["weight_bytes"] / (peaks["hbm_gbs"] * 1e9) * 1e6
+        tensor_time = st["padded_flops"] / (fp8_peak * 1e12) * 1e6
+        bound = "hbm" if hbm_time >= tensor_time else "tensor"
+        ffn_us = kern_us["grouped_ffn"]
+        if bound == "hbm":
+            achieved = st["weight_bytes"] / (ffn_us * 1e-6) / 1e9             # bytes: 3*d*f per activated instance
+            roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
+                        frac=achieved / peaks["hbm_gbs"], traffic=ncu_traffic_bytes(self.name),
+                        peak_source=peaks["source"] + " HBM copy (MEASURED_PEAKS.json)")
+        else:
+            achieved = st["padded_flops"] / (ffn_us * 1e-6) / 1e12            # flops: 6*d*f per padded row
+            roof = dict(bound="tensor", achieved=achieved, peak=fp8_peak, unit="TFLOP/s", frac=achieved / fp8_peak,
+                        traffic=ncu_traffic_bytes(self.name),
+                        peak_source=f"{primary}: " + (fp8["how"] if primary.startswith("fp8_measured") else
+                                                      peaks["source"] + " bf16 GEMM rate x 2 (nominal fp8/bf16 ratio)"),
+                        frac_vs={k: achieved / v for k, v in denoms.items()})
+        roof.update(kernel="ffn_kernel (gate/up + SwiGLU + down, one launch)", kernel_us=ffn_us)
+        block = {"weight_us": hbm_time, "padded_flop_us": tensor_time, "bound": bound,
+                 "frac": max(hbm_time, tensor_time) / us_step, "ffn_frac": max(hbm_time, tensor_time) / ffn_us,
+                 "tensor_peak": primary}
+        if bound == "tensor":
+            block["frac_vs"] = {k: max(hbm_time, st["padded_flops"] / (v * 1e12) * 1e6) / us_step
+                                for k, v in denoms.items()}
+        return roof, block
+
+
+def measure_e2e(torch, B, leg, K, warmup, barrier):
+    """Host buffers in, host result out, every step: two sets of device buffers and three streams, as a serving
+    loop would run it (step i+1's inputs come in and step i-1's result goes out while step i computes), captured
+    into CUDA graphs of `ce` steps, copies included.  Every step pays its own copies inside the timed region."""
+    wl, buf, pools, n_pools, max_m = leg.wl, leg.buf, leg.pools, leg.n_pools, leg.max_m
     h_ids = torch.from_numpy(wl.topk_ids).pin_memory()
     h_w = torch.from_numpy(wl.topk_w).pin_memory()
     h_x = torch.from_numpy(wl.x).to(torch.bfloat16).pin_memory()
     h_out = [torch.empty(wl.T, wl.d, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
     h2d = h_ids.numel() * 4 + h_w.numel() * 4 + h_x.numel() * 2
     d2h = h_out[0].numel() * 2
-    # Two sets of device buffers and three streams, as a serving loop would run it: step i+1's inputs come in
-    # and step i-1's result goes out while step i computes.  Every step still pays its own copies inside the
-    # timed region; PCIe carries both directions at once.
     buf2 = B.RankBuffers.for_workload(wl, M_cap=buf.M_cap, with_weights=False)
-    run_fn2 = (lambda packed: buf2.run_block_masked(max_m, packed=packed)) if max_m else None
-    sets = [(buf, graphs), (buf2, _capture_graphs(torch, buf2, pools, run_fn2))]
-    s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
-    ev_in = [torch.cuda.Event() for _ in range(2)]
-    ev_cmp = [torch.cuda.Event() for _ in range(2)]
-    ev_out = [torch.cuda.Event() for _ in range(2)]
+    sets = [buf, buf2]
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
 
-    def e2e_step(i):
-        j = i & 1
-        b, gs = sets[j]
-        with torch.cuda.stream(s_in):
-            s_in.wait_event(ev_cmp[j])                  # this set's previous step has read its inputs
-            b.topk_ids.copy_(h_ids, non_blocking=True)
-            b.topk_w.copy_(h_w, non_blocking=True)
-            b.x.copy_(h_x, non_blocking=True)
-            ev_in[j].record(s_in)
-        with torch.cuda.stream(s_cmp):
-            s_cmp.wait_event(ev_in[j])                  # the inputs are there
-            s_cmp.wait_event(ev_out[j])                 # and the previous result of this set has left
-            gs[i % n_pools].replay()
-            ev_cmp[j].record(s_cmp)
-        with torch.cuda.stream(s_out):
-            s_out.wait_event(ev_cmp[j])
-            h_out[j].copy_(b.out, non_blocking=True)
-            ev_out[j].record(s_out)
-
-    # The same pipeline captured once: a graph of `ce` consecutive steps over the three streams (every step's
-    # copies are nodes of the graph), so the host issues one launch per `ce` steps and its timing drops out.
-    def capture_e2e(ce):
+    def capture(ce):
         g = torch.cuda.CUDAGraph()
         gi = [torch.cuda.Event() for _ in range(ce)]
         gc = [torch.cuda.Event() for _ in range(ce)]
@@ -363,7 +460,7 @@ def run_gpu(args):
             s_in.wait_stream(cur)
             s_out.wait_stream(cur)
             for i in range(ce):
-                b = sets[i & 1][0]
+                b = sets[i & 1]
                 with torch.cuda.stream(s_in):
                     if i >= 2:
                         s_in.wait_event(gc[i - 2])     # this set's previous step has read its inputs
@@ -387,114 +484,54 @@ def run_gpu(args):
             cur.wait_stream(s_out)
         return g
 
-    Ke = min(K, 480)
-    ce = 2 * n_pools * max(1, 24 // n_pools)               # steps per captured graph (even: the buffer sets alternate)
-    for i in range(min(Wm, 5) + 1):
-        e2e_step(i)
-    barrier()
-    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    if Ke >= ce:
-        g_e2e = capture_e2e(ce)
+    Ke = max(2, min(K, 480))
+    ce = min(2 * n_pools * max(1, 24 // n_pools), (Ke // 2) * 2)     # steps per graph, even: the buffer sets alternate
+    # warm the launch path of the second buffer set outside capture
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        buf2.run_block_masked(max_m, packed=pools[0]) if max_m else buf2.run_block(packed=pools[0])
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g_e2e = capture(ce)
+    for _ in range(max(1, min(warmup, 3))):
         g_e2e.replay()
-        barrier()
-        Ke = (Ke // ce) * ce
-        f0.record()
-        for _ in range(Ke // ce):
-            g_e2e.replay()
-        f1.record()
-        e2e_mode = f"{ce} steps per CUDA graph, copies included"
-    else:
-        f0.record(s_in)
-        for i in range(Ke):
-            e2e_step(i)
-        f1.record(s_out)
-        e2e_mode = "launched step by step"
     barrier()
-    ms_e2e = f0.elapsed_time(f1) / Ke
-    e2e_ok = bool(torch.equal(h_out[0], h_out[1]) and torch.equal(h_out[0], buf.out.cpu()))
-
-    clocks = sampler.stop() if sampler is not None else None
-
-    ms_step, units = reduce_step(ms_total / K, float(st["G_act"]), "cuda" if world > 1 else None)
-    ms_e2e_max, _ = reduce_step(ms_e2e, float(st["G_act"]), "cuda" if world > 1 else None)
-    if world > 1:
-        dist.destroy_process_group()
-    if rank != 0:
-        return
-
-    peaks = _peaks()
-    us_step = ms_step * 1e3
-    hbm_time = st["weight_bytes"] / (peaks["hbm_gbs"] * 1e9) * 1e6
-    fp8_peak = peaks["bf16_tflops_sustained"] * NOMINAL_FP8_OVER_BF16
-    tensor_time = st["padded_flops"] / (fp8_peak * 1e12) * 1e6
-    bound = "hbm" if hbm_time >= tensor_time else "tensor"
-    # dominant kernel: the fused FFN kernel (both GEMMs of every activated instance in one launch)
-    ffn_us = kern_us["grouped_ffn"]
-    if bound == "hbm":
-        alg = st["weight_bytes"]                                   # bytes: 3*d*f per activated instance
-        achieved = alg / (ffn_us * 1e-6) / 1e9
-        roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s",
-                    frac=achieved / peaks["hbm_gbs"], traffic=NCU_TRAFFIC_BYTES.get(args.workload))
-    else:
-        alg = st["padded_flops"]                                   # flops: 6*d*f per padded row
-        achieved = alg / (ffn_us * 1e-6) / 1e12
-        roof = dict(bound="tensor", achieved=achieved, peak=fp8_peak, unit="TFLOP/s", frac=achieved / fp8_peak,
-                    traffic=NCU_TRAFFIC_BYTES.get(args.workload))
-    roof.update(kernel="ffn_kernel (gate/up + SwiGLU + down, one launch)", kernel_us=ffn_us, peak_source=peaks["source"] +
-                (" HBM copy" if bound == "hbm" else " bf16 sustained x 2 (nominal fp8/bf16 ratio)"))
-
-    out = {
-        "metric": METRIC, "value": us_step / units, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-        "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
-        "data": "synthetic",
-        "config": {"workload": args.workload, "T": wl.T, "top_k": wl.k, "E": wl.E, "d": wl.d, "f": wl.f,
-                   "G_act": st["G_act"], "N_local": st["N_local"], "M_pad": st["M_pad"],
-                   "layout": f"masked, max_m={max_m}" if max_m else "grouped",
-                   "graph": f"{chain_steps} consecutive steps per CUDA graph (weight copies in rotation), single-step graphs for the remainder",
-                   "l2": f"weights rotate through {n_pools} copies ({n_pools * weight_bytes_all / 1e9:.2f} GB >> L2)",
-                   "parallelism": f"{world} independent rank(s), no collective"},
-        "block_us": us_step, "tokens_per_s": st["n_valid"] * world / (us_step * 1e-6),
-        "block_roofline": {"weight_us": hbm_time, "padded_flop_us": tensor_time,
-                           "frac": max(hbm_time, tensor_time) / us_step,
-                           "ffn_frac": max(hbm_time, tensor_time) / kern_us["grouped_ffn"]},
-        "kernel_us": kern_us, "gpu_launches": 4 * K, "device_status": status,
-        "roofline": roof, "clocks": clocks,
-        "e2e": {"value": ms_e2e_max * 1e3 / units, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "pipeline": "two buffer sets, copy-in / compute / copy-out streams; " + e2e_mode, "steps": Ke,
-                "results_identical": e2e_ok},
-    }
-    if world == 1 and not args.no_cpu_baseline:
-        v, sample = oracle_sample_us_per_block(wl, budget_s=12.0)
-        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "sample": sample}
-    print(json.dumps(out))
+    Ke = (Ke // ce) * ce
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record()
+    for _ in range(Ke // ce):
+        g_e2e.replay()
+    f1.record()
+    barrier()
+    ms = f0.elapsed_time(f1) / Ke
+    ok = bool(torch.equal(h_out[0], h_out[1]) and torch.equal(h_out[0], buf.out.cpu()))
+    del buf2
+    return dict(ms=ms, steps=Ke, h2d=h2d, d2h=d2h, identical=ok,
+                mode=f"two buffer sets, copy-in / compute / copy-out streams; {ce} steps per CUDA graph, copies included")
 
 
-# --------------------------------------------------------------------------------------------------
-# cost-profile sweep (config 5) and fit
-# --------------------------------------------------------------------------------------------------
-
-def run_sweep(args):
-    import torch
-    from paper_2608_13057_b200 import binding as B
-    from paper_2608_13057_b200 import costmodel as C
+def sweep_rows(torch, B, Gs, Ns, replays, variant="fp8", device_weights=False, log=None):
+    """(G, N) points of config 5: G instances of the Qwen3-235B expert shape with N rows each; per point the
+    median / p10 / p90 over `replays` single-step graph replays of the whole block and of the FFN kernel alone."""
     from paper_2608_13057_b200 import workloads as W
-
-    torch.cuda.set_device(0)
     d, f = 4096, 1536
-    Gs = [int(g) for g in args.sweep_G.split(",")] if args.sweep_G else list(W.SWEEP_G)
-    Ns = [int(n) for n in args.sweep_N.split(",")] if args.sweep_N else list(W.SWEEP_N)
-    replays = args.replays
+    bf16 = variant == "bf16"
     rows = []
     gen = torch.Generator(device="cuda").manual_seed(4)
     for G in Gs:
-        # one weight set per G, copied into a rotation pool >> L2
-        wl0 = W.config5_point(G, 1, with_x=False)
+        wl0 = W.config5_point(G, 1, with_x=False)        # one weight set per G, copied into a rotation pool >> L2
         probe = B.RankBuffers(G, 1, G, G, 1, d, f)
-        bf16 = args.variant == "bf16"
-        packed = probe.pack_weights_bf16(*wl0.slot_weights_bf16()) if bf16 else probe.pack_weights(*wl0.slot_weights())
-        n_pools = min(64, max(2, math.ceil((1 << 30) / packed.numel())))
+        if bf16:
+            packed = probe.pack_weights_bf16(*wl0.slot_weights_bf16())
+        elif device_weights:
+            packed = probe.pack_weights(*W.slot_weights_cuda(wl0))
+        else:
+            packed = probe.pack_weights(*wl0.slot_weights())
+        n_pools = n_pools_for(packed.numel())
         pools = [packed] + [packed.clone() for _ in range(n_pools - 1)]
         del probe
+        torch.cuda.empty_cache()
         for N in Ns:
             T = G * N
             buf = B.RankBuffers(T, 1, G, G, 1, d, f)
@@ -505,7 +542,7 @@ def run_sweep(args):
             buf.x.copy_(torch.randn(T, d, generator=gen, device="cuda").to(torch.bfloat16))
             if bf16:
                 buf.alloc_bf16()
-            graphs = _capture_graphs(torch, buf, pools, buf.run_block_bf16 if bf16 else None)
+            graphs = _capture_graphs(torch, pools, buf.run_block_bf16 if bf16 else buf.run_block)
             s = buf.shape
             ffn_graphs = []
             for blob in pools:
@@ -537,34 +574,170 @@ def run_sweep(args):
             tiles = G * (-(-N // 128))
             rows.append(dict(G=G, n=N, N=G * N, tiles=tiles, t_block_us=t_block, t_ffn_us=t_ffn, block_p10=b10,
                              block_p90=b90, ffn_p10=f10, ffn_p90=f90, status=int(buf.status.item())))
-            print(json.dumps(rows[-1]), file=sys.stderr, flush=True)
+            if log is not None:
+                print(json.dumps(rows[-1]), file=log, flush=True)
             del buf, graphs, ffn_graphs
             torch.cuda.empty_cache()
         del pools, packed
         torch.cuda.empty_cache()
+    return rows
+
+
+def fit_rows(rows):
+    from paper_2608_13057_b200 import costmodel as C
     G = np.array([r["G"] for r in rows])
     N = np.array([r["N"] for r in rows])
     tiles = np.array([r["tiles"] for r in rows])
-    result = {"sweep": {"d": d, "f": f, "points": len(rows), "replays": replays, "variant": args.variant}, "rows": rows}
+    out = {}
     for scope in ("ffn", "block"):
         t = np.array([r[f"t_{scope}_us"] for r in rows])
-        result[f"fit_{scope}"] = C.fit_max_affine(G, N, t)
-        result[f"fit_{scope}_tile"] = C.fit_max_affine(G, N, t, tiles=tiles, tile_aware=True)
+        out[f"fit_{scope}"] = C.fit_max_affine(G, N, t)
+        out[f"fit_{scope}_tile"] = C.fit_max_affine(G, N, t, tiles=tiles, tile_aware=True)
+    return out
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2608_13057_b200 import binding as B
+    from paper_2608_13057_b200.ranks import reduce_step
+
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    K, Wm, R = args.steps, args.warmup, max(1, args.replays)
+    wl = make_workload(args.workload, rank)
+    leg = Leg(torch, B, args.workload, wl, max_m=args.max_m)
+    st = leg.st
+    sampler = ClockSampler(local) if rank == 0 else None
+
+    # ---- region A: R timed regions of exactly K steps each, inputs resident in HBM ------------------
+    ms_regions = leg.time_regions(K, Wm, R, barrier)
+    status = int(leg.buf.status.item())
+    # ---- region B: per-kernel durations ---------------------------------------------------------------
+    kern_us = leg.kernel_pass(min(K, 200))
+    # ---- e2e ------------------------------------------------------------------------------------------------
+    e2e = measure_e2e(torch, B, leg, K, Wm, barrier)
+    clocks = sampler.stop() if sampler is not None else None
+
+    step_ms = [m / K for m in ms_regions]
+    ms_step, units = reduce_step(float(np.median(step_ms)), float(st["G_act"]), "cuda" if world > 1 else None)
+    ms_e2e_max, _ = reduce_step(e2e["ms"], float(st["G_act"]), "cuda" if world > 1 else None)
+
+    extras = world == 1 and not args.no_extras and args.workload == "cfg2" and not args.max_m
+    linear = fit = fp8 = None
+    if extras:
+        del leg.graphs, leg.chain, leg.pools
+        torch.cuda.empty_cache()
+        # ---- the tensor-bound regime: config 4, the largest single-GPU configuration -----------------------
+        wl4 = make_workload("cfg4", 0)
+        leg4 = Leg(torch, B, "cfg4", wl4, device_weights=True)
+        sampler4 = ClockSampler(local)
+        K4 = leg4.chain_steps
+        ms4 = leg4.time_regions(K4, 3, R, barrier)
+        kern4 = leg4.kernel_pass(24)
+        clocks4 = sampler4.stop()
+        status4 = int(leg4.buf.status.item())
+        linear = dict(leg=leg4, ms=ms4, K=K4, kern=kern4, clocks=clocks4, status=status4)
+        # ---- reduced cost-profile sweep -> fit ------------------------------------------------------------------
+        rows = sweep_rows(torch, B, FIT_G, FIT_N, max(10, min(R, 30)), device_weights=True)
+        fit = dict(rows=rows, **fit_rows(rows))
+        # ---- dense fp8 GEMM rate of the vendor library, as a denominator -------------------------------------
+        fp8 = measure_fp8_peak(torch)
+    if world > 1:
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+
+    peaks = _peaks()
+    us_step = ms_step * 1e3
+    roof, block = leg.rooflines(us_step, kern_us, peaks, fp8)
+    pct = _pct([m * 1e3 for m in step_ms])
+    out = {
+        "metric": METRIC, "value": us_step / units, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
+        "data": "synthetic",
+        "config": workload_config(args.workload, wl, st, world, args.max_m),
+        "timing": {"regions": R, "steps_per_region": K, "statistic": "median over regions of (region time / K)",
+                   "graph": f"{leg.chain_steps} consecutive steps per CUDA graph (weight copies in rotation), "
+                            "single-step graphs for the remainder"},
+        "block_us": us_step, "block_us_percentiles": pct, "tokens_per_s": st["n_valid"] * world / (us_step * 1e-6),
+        "block_roofline": block, "kernel_us": kern_us, "gpu_launches": 4 * K, "device_status": status,
+        "roofline": roof, "clocks": clocks,
+        "e2e": {"value": ms_e2e_max * 1e3 / units, "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
+                "d2h_bytes_per_step": e2e["d2h"], "pipeline": e2e["mode"], "steps": e2e["steps"],
+                "results_identical": e2e["identical"]},
+    }
+    if extras:
+        l4 = linear["leg"]
+        step4 = [m / linear["K"] * 1e3 for m in linear["ms"]]
+        us4 = float(np.median(step4))
+        roof4, block4 = l4.rooflines(us4, linear["kern"], peaks, fp8)
+        out["regimes"] = {
+            "flat": {"workload": args.workload, "block_us": us_step, "bound": block["bound"], "block_frac": block["frac"],
+                     "ffn_frac": roof["frac"]},
+            "linear": {"workload": "cfg4", "config": workload_config("cfg4", l4.wl, l4.st, 1),
+                       "weights": "drawn on the device (same distribution and scale rule; timing only)",
+                       "value": us4 / l4.st["G_act"], "unit": UNIT, "block_us": us4, "block_us_percentiles": _pct(step4),
+                       "steps_per_region": linear["K"], "regions": R, "tokens_per_s": l4.st["n_valid"] / (us4 * 1e-6),
+                       "kernel_us": linear["kern"], "roofline": roof4, "block_roofline": block4,
+                       "clocks": linear["clocks"], "device_status": linear["status"]},
+        }
+        keep = ("a", "b", "b2", "c", "beta", "n_star", "fit_err", "n_flat", "n_linear")
+        out["fit"] = {"grid": {"G": list(FIT_G), "N_per_instance": list(FIT_N), "d": 4096, "f": 1536,
+                               "replays": max(10, min(R, 30))},
+                      "n_star": fit["fit_ffn_tile"]["n_star"],
+                      **{k: {kk: fit[k][kk] for kk in keep} for k in ("fit_ffn", "fit_ffn_tile", "fit_block", "fit_block_tile")},
+                      "points": [{k: r[k] for k in ("G", "n", "t_ffn_us", "t_block_us")} for r in fit["rows"]]}
+        out["measured_fp8"] = fp8
+    if world == 1 and not args.no_cpu_baseline:
+        v, sample = oracle_sample_us_per_block(wl, budget_s=12.0)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "sample": sample}
+    print(json.dumps(out))
+
+
+# --------------------------------------------------------------------------------------------------
+# cost-profile sweep (config 5) and fit
+# --------------------------------------------------------------------------------------------------
+
+def run_sweep(args):
+    import torch
+    from paper_2608_13057_b200 import binding as B
+    from paper_2608_13057_b200 import workloads as W
+
+    torch.cuda.set_device(0)
+    Gs = [int(g) for g in args.sweep_G.split(",")] if args.sweep_G else list(W.SWEEP_G)
+    Ns = [int(n) for n in args.sweep_N.split(",")] if args.sweep_N else list(W.SWEEP_N)
+    rows = sweep_rows(torch, B, Gs, Ns, args.replays, args.variant, device_weights=args.variant == "fp8", log=sys.stderr)
+    result = {"sweep": {"d": 4096, "f": 1536, "points": len(rows), "replays": args.replays, "variant": args.variant},
+              "rows": rows}
+    result.update(fit_rows(rows))
     print(json.dumps(result))
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the linear-regime leg, the in-run fit and the fp8 GEMM rate of the default line")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--sweep-G", default="")
     ap.add_argument("--sweep-N", default="")
-    ap.add_argument("--replays", type=int, default=30)
+    ap.add_argument("--replays", type=int, default=30, help="timed regions of K steps each (sweep: replays per point)")
     ap.add_argument("--variant", default="fp8", choices=["fp8", "bf16"], help="--sweep only: which steps 2 and 3")
     ap.add_argument("--max-m", type=int, default=0, help="> 0: run the block in the masked layout with this row stride")
     args = ap.parse_args()

@@ -145,6 +145,36 @@ def draw_expert_weights_bf16(weight_seed: int, e: int, d: int, f: int, std: floa
     return (w13.to(torch.bfloat16).to(torch.float32).numpy(), w2.to(torch.bfloat16).to(torch.float32).numpy())
 
 
+def slot_weights_cuda(wl: "Workload", device="cuda", std: float = 0.02):
+    """Per-slot weights drawn and quantised ON THE DEVICE, for timing-only runs of the large shapes (the numpy
+    draws above take minutes for config 4 and the sweep): same distribution, layout and scale rule as
+    draw_expert_weights, other random numbers, so results made with them are not comparable with the oracle's.
+    Replica slots of one expert get identical copies.  Returns torch tensors (w13_q u8 [G,2f,d], w13_s f32
+    [G,2f/128,d/128], w2_q u8 [G,d,f], w2_s f32 [G,d/128,f/128])."""
+    dev = torch.device(device)
+    G, d, f = wl.G_max, wl.d, wl.f
+    w13_q = torch.zeros(G, 2 * f, d, dtype=torch.uint8, device=dev)
+    w13_s = torch.ones(G, 2 * f // 128, d // 128, dtype=torch.float32, device=dev)
+    w2_q = torch.zeros(G, d, f, dtype=torch.uint8, device=dev)
+    w2_s = torch.ones(G, d // 128, f // 128, dtype=torch.float32, device=dev)
+
+    def quant(w):
+        R, C = w.shape
+        blk = w.reshape(R // 128, 128, C // 128, 128)
+        s = _pow2_block_scale(blk.abs().amax(dim=(1, 3)))
+        q = (blk / s[:, None, :, None]).to(torch.float8_e4m3fn)
+        return q.reshape(R, C).view(torch.uint8), s
+
+    for i in range(G):
+        e = int(wl.slot_expert[i])
+        if e < 0:
+            continue
+        gen = torch.Generator(device=dev).manual_seed(int(wl.weight_seed) * 1000003 + e)
+        w13_q[i], w13_s[i] = quant(torch.randn(2 * f, d, generator=gen, device=dev) * std)
+        w2_q[i], w2_s[i] = quant(torch.randn(d, f, generator=gen, device=dev) * std)
+    return w13_q, w13_s, w2_q, w2_s
+
+
 def draw_activations(seed: int, T: int, d: int) -> np.ndarray:
     x = _rng(seed, _TAG_X).standard_normal((T, d), dtype=np.float32)
     return torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
