@@ -317,9 +317,10 @@ def tensor_denominators(peaks, fp8):
 class Leg:
     """One workload on the device: buffers, weight copies, graphs, and the timed regions."""
 
-    def __init__(self, torch, B, name, wl, max_m=0, device_weights=False):
+    def __init__(self, torch, B, name, wl, max_m=0, device_weights=False, path="permute"):
         from paper_2608_13057_b200 import workloads as W
         self.torch, self.B, self.name, self.wl, self.max_m = torch, B, name, wl, max_m
+        self.path = "permute" if max_m else path         # "gather": tempo_quantize_tokens + tempo_grouped_ffn_gather
         self.st = workload_stats(wl)
         M_cap = wl.G_max * max_m if max_m else None
         if device_weights:
@@ -331,10 +332,15 @@ class Leg:
         buf = self.buf
         self.n_pools = n_pools_for(buf.packed.numel())
         self.pools = [buf.packed] + [buf.packed.clone() for _ in range(self.n_pools - 1)]
-        self.run = (lambda packed: buf.run_block_masked(max_m, packed=packed)) if max_m else buf.run_block
+        self.run = self.runner(buf)
         self.graphs = _capture_graphs(torch, self.pools, self.run)
         self.chain_steps = self.n_pools * max(1, 12 // self.n_pools)
         self.chain = None
+
+    def runner(self, buf):
+        if self.max_m:
+            return lambda packed: buf.run_block_masked(self.max_m, packed=packed)
+        return buf.run_block_gather if self.path == "gather" else buf.run_block
 
     def replay_steps(self, K):
         """Exactly K steps: whole chains of `chain_steps` steps, then single-step graphs for the remainder."""
@@ -369,7 +375,8 @@ class Leg:
         """The same steps launched call by call with events between the kernels (queued behind a spin kernel so
         that no launch is late): per-kernel CUDA-event durations on the launching stream."""
         torch, B, buf, max_m = self.torch, self.B, self.buf, self.max_m
-        names = ["count_dispatch", "permute_pad", "grouped_ffn", "unpermute_combine"]
+        gather = self.path == "gather"
+        names = ["count_dispatch", "quantize_tokens" if gather else "permute_pad", "grouped_ffn", "unpermute_combine"]
         ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(Kb)]
         s = buf.shape
         torch.cuda._sleep(int(4e7))
@@ -391,11 +398,17 @@ class Leg:
                                        buf.counts, buf.inst_count, buf.inst_off, buf.pair_row, buf.row_pair,
                                        buf.tile_inst, buf.m_pad, buf.status)
                 ev[i][1].record()
-                B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status,
-                                    pair_row=buf.pair_row)
-                ev[i][2].record()
-                B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
-                                    buf.status, buf.workspace)
+                if gather:
+                    B.tempo_quantize_tokens(s, buf.x, buf.n_valid, buf.x_q, buf.x_sf, buf.status)
+                    ev[i][2].record()
+                    B.tempo_grouped_ffn_gather(s, buf.x_q, buf.x_sf, buf.row_pair, blob, buf.inst_off, buf.m_pad,
+                                               buf.h_q, buf.h_sf, buf.y, buf.status, buf.workspace)
+                else:
+                    B.tempo_permute_pad(s, buf.x, buf.row_pair, buf.m_pad, buf.a_q, buf.a_sf, buf.status,
+                                        pair_row=buf.pair_row)
+                    ev[i][2].record()
+                    B.tempo_grouped_ffn(s, buf.a_q, buf.a_sf, blob, buf.inst_off, buf.m_pad, buf.h_q, buf.h_sf, buf.y,
+                                        buf.status, buf.workspace)
             ev[i][3].record()
             B.tempo_unpermute_combine(s, buf.y, buf.pair_row, buf.topk_w, buf.n_valid, buf.out, buf.status)
             ev[i][4].record()
@@ -448,6 +461,7 @@ def measure_e2e(torch, B, leg, K, warmup, barrier):
     d2h = h_out[0].numel() * 2
     buf2 = B.RankBuffers.for_workload(wl, M_cap=buf.M_cap, with_weights=False)
     sets = [buf, buf2]
+    runs = [leg.runner(buf), leg.runner(buf2)]
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
 
     def capture(ce):
@@ -471,10 +485,7 @@ def measure_e2e(torch, B, leg, K, warmup, barrier):
                 cur.wait_event(gi[i])
                 if i >= 2:
                     cur.wait_event(go[i - 2])          # and its previous result has left
-                if max_m:
-                    b.run_block_masked(max_m, packed=pools[i % n_pools])
-                else:
-                    b.run_block(packed=pools[i % n_pools])
+                runs[i & 1](packed=pools[i % n_pools])
                 gc[i].record(cur)
                 with torch.cuda.stream(s_out):
                     s_out.wait_event(gc[i])
@@ -490,7 +501,7 @@ def measure_e2e(torch, B, leg, K, warmup, barrier):
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
-        buf2.run_block_masked(max_m, packed=pools[0]) if max_m else buf2.run_block(packed=pools[0])
+        runs[1](packed=pools[0])
     torch.cuda.current_stream().wait_stream(side)
     torch.cuda.synchronize()
     g_e2e = capture(ce)
@@ -616,7 +627,7 @@ def run_gpu(args):
 
     K, Wm, R = args.steps, args.warmup, max(1, args.replays)
     wl = make_workload(args.workload, rank)
-    leg = Leg(torch, B, args.workload, wl, max_m=args.max_m)
+    leg = Leg(torch, B, args.workload, wl, max_m=args.max_m, path=args.path)
     st = leg.st
     sampler = ClockSampler(local) if rank == 0 else None
 
@@ -640,7 +651,7 @@ def run_gpu(args):
         torch.cuda.empty_cache()
         # ---- the tensor-bound regime: config 4, the largest single-GPU configuration -----------------------
         wl4 = make_workload("cfg4", 0)
-        leg4 = Leg(torch, B, "cfg4", wl4, device_weights=True)
+        leg4 = Leg(torch, B, "cfg4", wl4, device_weights=True, path=args.path)
         sampler4 = ClockSampler(local)
         K4 = leg4.chain_steps
         ms4 = leg4.time_regions(K4, 3, R, barrier)
@@ -667,6 +678,7 @@ def run_gpu(args):
         "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3",
         "data": "synthetic",
         "config": workload_config(args.workload, wl, st, world, args.max_m),
+        "path": leg.path,
         "timing": {"regions": R, "steps_per_region": K, "statistic": "median over regions of (region time / K)",
                    "graph": f"{leg.chain_steps} consecutive steps per CUDA graph (weight copies in rotation), "
                             "single-step graphs for the remainder"},
@@ -739,6 +751,9 @@ def main():
     ap.add_argument("--sweep-N", default="")
     ap.add_argument("--replays", type=int, default=30, help="timed regions of K steps each (sweep: replays per point)")
     ap.add_argument("--variant", default="fp8", choices=["fp8", "bf16"], help="--sweep only: which steps 2 and 3")
+    ap.add_argument("--path", default="permute", choices=["permute", "gather"],
+                    help="steps 2-3: tempo_permute_pad + tempo_grouped_ffn, or tempo_quantize_tokens + "
+                         "tempo_grouped_ffn_gather (same results bit for bit)")
     ap.add_argument("--max-m", type=int, default=0, help="> 0: run the block in the masked layout with this row stride")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

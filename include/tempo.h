@@ -204,6 +204,28 @@ int tempo_grouped_ffn_bounded(const tempo_shape* shape, const void* a_q, const u
                               uint32_t* status, void* workspace, uint64_t wait_limit_ns, void* stream);
 
 /*
+ * Steps 2 and 3 with the gather fused into the GEMM (Appendix B counts "scatter/gather, quantization" among
+ * the un-fused per-token kernels that multiply the per-token slope at pipeline scope; this pair removes the
+ * permuted copy).  Same results as tempo_permute_pad + tempo_grouped_ffn, bit for bit.
+ *   tempo_quantize_tokens     x_q[t,:] = e4m3(x[t,:] / 2^eps) per 128-column block for every live token
+ *                             (t < n_valid), the rule of step 2; x_sf[t*S + kb] = eps + 127 (UE8M0), S =
+ *                             4*ceil((d/128)/4) bytes per token (tempo_token_sf_bytes gives T*S).  It reads
+ *                             nothing step 1 writes: enqueued right after tempo_count_dispatch on the same
+ *                             stream it runs beside it, and still finishes only after it.
+ *        in  x bf16 [T, d], n_valid (or NULL)      out  x_q u8 [T, d], x_sf u8 [T*S]
+ *   tempo_grouped_ffn_gather  tempo_grouped_ffn whose gate/up GEMM fetches row r of its operand from
+ *                             x_q[row_pair[r] / k, :] (rows with row_pair[r] < 0 are zero rows) while it fills
+ *                             its shared-memory stages: a_q / a_sf are never materialised.  Same `workspace`,
+ *                             waits and status bits as tempo_grouped_ffn.
+ */
+int tempo_token_sf_bytes(const tempo_shape* shape /*[host]*/, size_t* bytes /*[host]*/);
+int tempo_quantize_tokens(const tempo_shape* shape, const void* x_bf16, const int32_t* n_valid, void* x_q,
+                          uint8_t* x_sf, uint32_t* status, void* stream);
+int tempo_grouped_ffn_gather(const tempo_shape* shape, const void* x_q, const uint8_t* x_sf, const int32_t* row_pair,
+                             const void* packed, const int32_t* inst_off, const int32_t* m_pad, void* h_q,
+                             uint8_t* h_sf, void* y_bf16, uint32_t* status, void* workspace, void* stream);
+
+/*
  * tempo_grouped_ffn without a caller-provided scratch buffer.  (The paper has no counterpart: this
  * exists for the integration, not for the method.)  Some callers cannot allocate device memory at
  * the point where they need the FFN: code that runs after the serving process has frozen its

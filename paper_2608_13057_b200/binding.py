@@ -21,7 +21,8 @@ EXPORTS = (
     "tempo_version", "tempo_status_string", "tempo_m_cap_bound", "tempo_sf_bytes", "tempo_workspace_bytes",
     "tempo_packed_weight_bytes",
     "tempo_pack_weights", "tempo_count_dispatch", "tempo_count_dispatch_sampled", "tempo_permute_pad", "tempo_ffn_gate_up", "tempo_ffn_down",
-    "tempo_grouped_ffn", "tempo_grouped_ffn_bounded", "tempo_grouped_ffn_static", "tempo_unpermute_combine",
+    "tempo_grouped_ffn", "tempo_grouped_ffn_bounded", "tempo_grouped_ffn_static",
+    "tempo_token_sf_bytes", "tempo_quantize_tokens", "tempo_grouped_ffn_gather", "tempo_unpermute_combine",
     "tempo_count_dispatch_masked", "tempo_permute_pad_masked", "tempo_grouped_ffn_masked",
     "tempo_packed_weight_bytes_bf16", "tempo_pack_weights_bf16", "tempo_permute_pad_bf16", "tempo_grouped_ffn_bf16",
 )
@@ -161,6 +162,27 @@ def tempo_grouped_ffn(shape, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf
            "tempo_grouped_ffn")
 
 
+def tempo_token_sf_bytes(shape: TempoShape) -> int:
+    out = ctypes.c_size_t(0)
+    _check(_lib.tempo_token_sf_bytes(ctypes.byref(shape), ctypes.byref(out)), "tempo_token_sf_bytes")
+    return out.value
+
+
+def tempo_quantize_tokens(shape, x_bf16, n_valid, x_q, x_sf, status):
+    _check(_lib.tempo_quantize_tokens(ctypes.byref(shape), _ptr(x_bf16, torch.bfloat16), _ptr(n_valid, torch.int32),
+                                      _ptr(x_q, torch.uint8), _ptr(x_sf, torch.uint8), _ptr(status, torch.int32),
+                                      _stream()), "tempo_quantize_tokens")
+
+
+def tempo_grouped_ffn_gather(shape, x_q, x_sf, row_pair, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, workspace):
+    _check(_lib.tempo_grouped_ffn_gather(ctypes.byref(shape), _ptr(x_q, torch.uint8), _ptr(x_sf, torch.uint8),
+                                         _ptr(row_pair, torch.int32), _ptr(packed, torch.uint8),
+                                         _ptr(inst_off, torch.int32), _ptr(m_pad, torch.int32), _ptr(h_q, torch.uint8),
+                                         _ptr(h_sf, torch.uint8), _ptr(y_bf16, torch.bfloat16),
+                                         _ptr(status, torch.int32), _ptr(workspace, torch.uint8), _stream()),
+           "tempo_grouped_ffn_gather")
+
+
 def tempo_grouped_ffn_bounded(shape, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, workspace,
                               wait_limit_ns):
     _check(_lib.tempo_grouped_ffn_bounded(ctypes.byref(shape), _ptr(a_q, torch.uint8), _ptr(a_sf, torch.uint8),
@@ -278,6 +300,8 @@ class RankBuffers:
         self.y = torch.zeros(self.M_cap, d, dtype=torch.bfloat16, device=dev)
         self.out = torch.zeros(T, d, dtype=torch.bfloat16, device=dev)
         self.workspace = torch.zeros(tempo_workspace_bytes(self.shape), **u8)   # counters start at zero
+        self.x_q = torch.zeros(T, d, **u8)                  # per-token quantised activations (gather form)
+        self.x_sf = torch.full((tempo_token_sf_bytes(self.shape),), 127, **u8)
         self.packed = None
 
     def pack_weights(self, w13_q, w13_s, w2_q, w2_s):
@@ -299,6 +323,19 @@ class RankBuffers:
         tempo_permute_pad(s, self.x, self.row_pair, self.m_pad, self.a_q, self.a_sf, self.status, pair_row=self.pair_row)
         tempo_grouped_ffn(s, self.a_q, self.a_sf, packed, self.inst_off, self.m_pad, self.h_q, self.h_sf, self.y,
                           self.status, self.workspace)
+        tempo_unpermute_combine(s, self.y, self.pair_row, self.topk_w, self.n_valid, self.out, self.status)
+
+    def run_block_gather(self, packed=None):
+        """The same block with the gather fused into the FFN: quantise tokens (beside the dispatch), then the
+        FFN fetches its rows by row_pair.  Same results bit for bit; a_q / a_sf are not written."""
+        s = self.shape
+        packed = self.packed if packed is None else packed
+        tempo_count_dispatch(s, self.topk_ids, self.n_valid, self.replica_map, self.quota, self.cum_counts,
+                             self.counts, self.inst_count, self.inst_off, self.pair_row, self.row_pair,
+                             self.tile_inst, self.m_pad, self.status)
+        tempo_quantize_tokens(s, self.x, self.n_valid, self.x_q, self.x_sf, self.status)
+        tempo_grouped_ffn_gather(s, self.x_q, self.x_sf, self.row_pair, packed, self.inst_off, self.m_pad, self.h_q,
+                                 self.h_sf, self.y, self.status, self.workspace)
         tempo_unpermute_combine(s, self.y, self.pair_row, self.topk_w, self.n_valid, self.out, self.status)
 
     def run_block_masked(self, max_m, packed=None):

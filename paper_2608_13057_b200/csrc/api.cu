@@ -56,6 +56,9 @@ static bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Scale bytes per token of the per-token quantised activations: one per 128 columns, rounded up to 4.
+static int token_sf_stride(int d) { return 4 * (((d / 128) + 3) / 4); }
+
 static int sm_count() {
   int dev = 0, n = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
@@ -67,14 +70,17 @@ static int sm_count() {
 static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,
                            const int32_t* inst_off, const int32_t* m_pad, void* h_q, uint8_t* h_sf, void* y,
                            uint32_t* status, void* workspace, cudaStream_t stream, int max_m = 0,
-                           const int32_t* inst_count = nullptr, unsigned long long wait_ns = kDefaultWaitNs) {
+                           const int32_t* inst_count = nullptr, unsigned long long wait_ns = kDefaultWaitNs,
+                           const uint8_t* x_q = nullptr, const uint8_t* x_sf = nullptr, const int32_t* row_pair = nullptr) {
   const PackLayout L = pack_layout(s->G_max, s->d, s->f);
   const uint8_t* blob = static_cast<const uint8_t*>(packed);
   const int sms = sm_count();
   if (sms <= 0) return TEMPO_ERR_CUDA;
   CUtensorMap tmA1, tmA2, tmY;
   // a side that does not run still needs a well-formed map; point it at a buffer that exists
-  if (!make_map(&tmA1, (run_mask & 1) ? a_q : h_q, s->M_cap, (run_mask & 1) ? s->d : s->f, 128)) return TEMPO_ERR_CUDA;
+  const bool gather = x_q != nullptr;              // gate/up rows fetched from the per-token buffers: no a_q
+  if (!make_map(&tmA1, (run_mask & 1) && !gather ? a_q : h_q, s->M_cap, (run_mask & 1) && !gather ? s->d : s->f, 128))
+    return TEMPO_ERR_CUDA;
   if (!make_map(&tmA2, h_q, s->M_cap, s->f, 128)) return TEMPO_ERR_CUDA;
   // Y stores: 32-row x 128-byte boxes (bf16 seen as bytes: 2d per row)
   if (!make_map(&tmY, (run_mask & 2) ? y : h_q, s->M_cap, (run_mask & 2) ? 2ull * s->d : s->f, 32)) return TEMPO_ERR_CUDA;
@@ -98,6 +104,15 @@ static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, 
   p.done = p.ready ? p.ready + s->M_cap / 128 : nullptr;
   p.status = status;
   p.wait_ns = wait_ns;
+  if (gather) {
+    p.x_q = x_q;
+    p.x_sf = x_sf;
+    p.row_pair = row_pair;
+    p.x_sf_stride = token_sf_stride(s->d);
+    p.k = s->k;
+    p.T = s->T;
+    return launch_ffn_gather(tmA2, tmY, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+  }
   return launch_ffn(tmA1, tmA2, tmY, p, sms, stream) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
 }
 
@@ -251,6 +266,36 @@ int tempo_grouped_ffn(const tempo_shape* s, const void* a_q, const uint8_t* a_sf
     return TEMPO_ERR_NULL;
   return launch_ffn_host(3, s, a_q, a_sf, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, workspace,
                          static_cast<cudaStream_t>(stream));
+}
+
+int tempo_token_sf_bytes(const tempo_shape* s, size_t* bytes) {
+  if (bytes == nullptr) return TEMPO_ERR_NULL;
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  *bytes = static_cast<size_t>(s->T) * token_sf_stride(s->d);
+  return TEMPO_OK;
+}
+
+int tempo_quantize_tokens(const tempo_shape* s, const void* x_bf16, const int32_t* n_valid, void* x_q, uint8_t* x_sf,
+                          uint32_t* status, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!x_bf16 || !x_q || !x_sf || !status) return TEMPO_ERR_NULL;
+  QuantizeParams p{s->T, s->d, token_sf_stride(s->d), static_cast<const __nv_bfloat16*>(x_bf16), n_valid,
+                   static_cast<uint8_t*>(x_q), x_sf};
+  return launch_quantize_tokens(p, sm_count(), static_cast<cudaStream_t>(stream)) == cudaSuccess ? TEMPO_OK : TEMPO_ERR_CUDA;
+}
+
+int tempo_grouped_ffn_gather(const tempo_shape* s, const void* x_q, const uint8_t* x_sf, const int32_t* row_pair,
+                             const void* packed, const int32_t* inst_off, const int32_t* m_pad, void* h_q,
+                             uint8_t* h_sf, void* y_bf16, uint32_t* status, void* workspace, void* stream) {
+  const int rc = check_shape(s);
+  if (rc != TEMPO_OK) return rc;
+  if (!x_q || !x_sf || !row_pair || !packed || !inst_off || !m_pad || !h_q || !h_sf || !y_bf16 || !status || !workspace)
+    return TEMPO_ERR_NULL;
+  return launch_ffn_host(3, s, nullptr, nullptr, packed, inst_off, m_pad, h_q, h_sf, y_bf16, status, workspace,
+                         static_cast<cudaStream_t>(stream), 0, nullptr, kDefaultWaitNs, static_cast<const uint8_t*>(x_q),
+                         x_sf, row_pair);
 }
 
 int tempo_grouped_ffn_bounded(const tempo_shape* s, const void* a_q, const uint8_t* a_sf, const void* packed,

@@ -42,13 +42,24 @@ constexpr int kStages = 4;
 constexpr int kStageBytes = kABytes + kBBytes + 2048;     // 51200, a multiple of 1024
 constexpr int kGemmThreads = 384;
 constexpr int kEpiWarp0 = 4;                               // first of the 8 epilogue warps
+constexpr int kGatherWarp0 = 12;                           // gather form: 4 more warps, one per 32 rows of the A tile
+constexpr int kGatherThreads = 512;
 constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 4 * kStoreBytes + 1024;
 
 // kBf16 = false: the fp8 path described above.  kBf16 = true: the bf16 variant (the paper calibrates a
 // bf16 grouped GEMM beside the fp8 one, Section 2.1): the same ring, roles and tiles with 64 bf16
 // values per 128-byte K-block, tcgen05.mma.kind::f16 without scales, and H stored as bf16.
-template <bool kBf16>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+//
+// kGather = true (fp8 only): the gate/up operand is not read from a permuted copy.  Four more warps
+// (12-15) fetch each row of the A tile from the per-token quantised activations x_q by the row's
+// token (row_pair / k) with 16-byte cp.async copies straight into the 128-byte-swizzled stage, and its
+// scale bytes from x_sf into the stage's scale atom; rows without a pair are zero-filled.  That takes
+// the permuted a_q / a_sf buffers (one write and NT re-reads of every row) out of the block.  The
+// stage's "full" barrier then counts five arrivals (weights + four gather warps) instead of two; on
+// down tiles the activation producer makes up the difference.  512 threads leave 128 registers per
+// thread at launch; the producer and gather warps hand most of theirs to the epilogue warps (setmaxnreg).
+template <bool kBf16, bool kGather>
+__global__ void __launch_bounds__(kGather ? kGatherThreads : kGemmThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
            const __grid_constant__ CUtensorMap tmY, const FfnParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -73,7 +84,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   pdl_trigger();
   // prologue that needs nothing from the previous kernel: barriers, tensor memory, descriptor fetch
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 2); mbar_init(smem_u32(&s_empty[s]), 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), kGather ? 5 : 2); mbar_init(smem_u32(&s_empty[s]), 1); }
     mbar_init(smem_u32(&s_acc_full), 1);
     mbar_init(smem_u32(&s_acc_empty), 8);
     s_abort_storage = 0;
@@ -111,7 +122,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   } else {
     const int m_pad_c = max(0, min(*p.m_pad, p.M_cap)) & ~(kTileM - 1);
 #pragma unroll 1
-    for (int i = tid; i <= G; i += kGemmThreads) s_toff[i] = max(0, min(p.inst_off[i], m_pad_c)) >> 7;
+    for (int i = tid; i <= G; i += static_cast<int>(blockDim.x)) s_toff[i] = max(0, min(p.inst_off[i], m_pad_c)) >> 7;
   }
   __syncthreads();
   const int m_tiles = s_toff[G];
@@ -142,53 +153,107 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   const uint32_t tmem_base = s_tmem_base;
   const int cold_tiles = s_cold[G], hot_tiles = m_tiles - cold_tiles;
   const TileOrder order1(p.side[0].NT, hot_tiles, cold_tiles, gridDim.x), order2(p.side[1].NT, hot_tiles, cold_tiles, gridDim.x);
-
-  if (warp == 0) {
-    // ------------------------------- weight producer ------------------------------------------
-    if (lane == 0) {
-      uint32_t stage = 0, phase = 0;
-      bool ok = true;
-      TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
-      int side, x;
-      while (ok && it.next(side, x)) {
-        const GemmSide& gs = p.side[side];
-        const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2, stride);
-        const uint8_t* sfb_src = gs.sfb + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.JK * kSfbBytes;
-        const uint8_t* b_src = gs.wt + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.Kb * kBBytes;
-        const bool stream_b = w.m_tiles <= 2;
+  // Roles by warpgroup (the register hand-over of the gather form works on whole warpgroups of four warps):
+  // 128 x (72 + 176 + 176 + 80) = 64512 of the SM's 65536 registers.
+  if (warp < kEpiWarp0) {
+    if constexpr (kGather) asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    if (warp == 0) {
+      // ------------------------------- weight producer ------------------------------------------
+      if (lane == 0) {
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+        int side, x;
+        while (ok && it.next(side, x)) {
+          const GemmSide& gs = p.side[side];
+          const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2, stride);
+          const uint8_t* sfb_src = gs.sfb + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.JK * kSfbBytes;
+          const uint8_t* b_src = gs.wt + (static_cast<size_t>(w.inst) * gs.NT + w.nt) * gs.Kb * kBBytes;
+          const bool stream_b = w.m_tiles <= 2;
 #pragma unroll 1
-        for (int kb = 0; kb < gs.Kb; ++kb) {
-          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
-          const uint32_t full = smem_u32(&s_full[stage]);
-          const uint32_t sB = smem_base + stage * kStageBytes + kABytes, sSF = sB + kBBytes;
-          const bool with_sf = !kBf16 && (kb & 3) == 0;
-          mbar_arrive_expect_tx(full, kBBytes + (with_sf ? kSfbBytes : 0));
-          if (stream_b) bulk_load_stream(sB, b_src + static_cast<size_t>(kb) * kBBytes, kBBytes, full);
-          else bulk_load(sB, b_src + static_cast<size_t>(kb) * kBBytes, kBBytes, full);
-          if (with_sf) bulk_load(sSF + kSfaBytes, sfb_src + static_cast<size_t>(kb >> 2) * kSfbBytes, kSfbBytes, full);
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          for (int kb = 0; kb < gs.Kb; ++kb) {
+            if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
+            const uint32_t full = smem_u32(&s_full[stage]);
+            const uint32_t sB = smem_base + stage * kStageBytes + kABytes, sSF = sB + kBBytes;
+            const bool with_sf = !kBf16 && (kb & 3) == 0;
+            mbar_arrive_expect_tx(full, kBBytes + (with_sf ? kSfbBytes : 0));
+            if (stream_b) bulk_load_stream(sB, b_src + static_cast<size_t>(kb) * kBBytes, kBBytes, full);
+            else bulk_load(sB, b_src + static_cast<size_t>(kb) * kBBytes, kBBytes, full);
+            if (with_sf) bulk_load(sSF + kSfaBytes, sfb_src + static_cast<size_t>(kb >> 2) * kSfbBytes, kSfbBytes, full);
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
         }
       }
-    }
-  } else if (warp == 2) {
-    // ------------------------------- activation producer --------------------------------------
-    if (lane == 0) {
-      uint32_t stage = 0, phase = 0;
-      int n_down = 0;
-      bool ok = true;
-      TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
-      int side, x;
-      while (ok && it.next(side, x)) {
-        const GemmSide& gs = p.side[side];
-        const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2, stride);
-        const uint8_t* sfa_src = gs.sfa + static_cast<size_t>(w.row0 >> 7) * gs.JK * kSfaBytes;
-        const CUtensorMap* tm = side == 0 ? &tmA1 : &tmA2;
-        if (side == 1 && fused) {
-          // wait until the scout (warp 3) has seen every H block of these 128 rows complete
-          ++n_down;
+    } else if (warp == 2) {
+      // ------------------------------- activation producer --------------------------------------
+      if (lane == 0) {
+        uint32_t stage = 0, phase = 0;
+        int n_down = 0;
+        bool ok = true;
+        TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+        int side, x;
+        while (ok && it.next(side, x)) {
+          const GemmSide& gs = p.side[side];
+          const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2, stride);
+          const uint8_t* sfa_src = gs.sfa + static_cast<size_t>(w.row0 >> 7) * gs.JK * kSfaBytes;
+          const CUtensorMap* tm = side == 0 ? &tmA1 : &tmA2;
+          if (kGather && side == 0) {                      // the gather warps fill these stages
+            const uint32_t adv = stage + static_cast<uint32_t>(gs.Kb);
+            phase ^= (adv / kStages) & 1u;
+            stage = adv % kStages;
+            continue;
+          }
+          if (side == 1 && fused) {
+            // wait until the scout (warp 3) has seen every H block of these 128 rows complete
+            ++n_down;
+            unsigned long long t0 = 0;
+            for (uint32_t spin = 0; *s_dep < n_down; ++spin) {
+              if ((spin & 255u) == 255u) {
+                if (*s_abort) { ok = false; break; }
+                const unsigned long long now = global_timer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > wait_ns) { *s_abort = 1; ok = false; break; }
+              }
+            }
+            if (!ok) break;
+            // The scout's acquire load saw the rows published; its word reaches this thread through
+            // shared memory (block-scope fences on both sides), then the proxy fence orders the
+            // ordinary stores that wrote H before the TMA reads below.
+            __threadfence_block();
+            asm volatile("fence.proxy.async;" ::: "memory");
+          }
+#pragma unroll 1
+          for (int kb = 0; kb < gs.Kb; ++kb) {
+            if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
+            const uint32_t full = smem_u32(&s_full[stage]);
+            const uint32_t sA = smem_base + stage * kStageBytes, sSF = sA + kABytes + kBBytes;
+            const bool with_sf = !kBf16 && (kb & 3) == 0;
+            mbar_arrive_expect_tx(full, kABytes + (with_sf ? kSfaBytes : 0));
+            if constexpr (kGather) mbar_arrive_n(full, 3);   // stands in for the gather warps, idle on down tiles
+            tma_load_2d(sA, tm, full, kb * kBlockK, w.row0);
+            if (with_sf) bulk_load(sSF, sfa_src + static_cast<size_t>(kb >> 2) * kSfaBytes, kSfaBytes, full);
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    } else if (warp == 3) {
+      // ------------------------------- dependency scout -----------------------------------------
+      // Runs ahead through this CTA's down tiles: waits (bounded) until the four epilogue warp pairs of
+      // every gate/up tile of the tile's 128 rows have published their H rows, then tells the
+      // activation producer through s_dep.  The last down tile of an M-tile to get here puts the
+      // two global counters back to zero, so the workspace is clean when the kernel ends.
+      if (lane == 0 && fused) {
+        TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+        int side, x, cleared = 0;
+        const int want = 4 * p.side[0].NT;
+        bool ok = true;
+        while (ok && it.next(side, x)) {
+          if (side == 0) continue;
+          const WorkItem w = decode_item(1, x, s_toff, s_cold, G, order2, stride);
+          const int tau = w.row0 >> 7;
           unsigned long long t0 = 0;
-          for (uint32_t spin = 0; *s_dep < n_down; ++spin) {
-            if ((spin & 255u) == 255u) {
+          for (uint32_t spin = 0; ld_acquire(p.ready + tau) < want; ++spin) {
+            if ((spin & 63u) == 63u) {
               if (*s_abort) { ok = false; break; }
               const unsigned long long now = global_timer_ns();
               if (t0 == 0) t0 = now;
@@ -196,100 +261,122 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
             }
           }
           if (!ok) break;
-          // The scout's acquire load saw the rows published; its word reaches this thread through
-          // shared memory (block-scope fences on both sides), then the proxy fence orders the
-          // ordinary stores that wrote H before the TMA reads below.
           __threadfence_block();
-          asm volatile("fence.proxy.async;" ::: "memory");
-        }
-#pragma unroll 1
-        for (int kb = 0; kb < gs.Kb; ++kb) {
-          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
-          const uint32_t full = smem_u32(&s_full[stage]);
-          const uint32_t sA = smem_base + stage * kStageBytes, sSF = sA + kABytes + kBBytes;
-          const bool with_sf = !kBf16 && (kb & 3) == 0;
-          mbar_arrive_expect_tx(full, kABytes + (with_sf ? kSfaBytes : 0));
-          tma_load_2d(sA, tm, full, kb * kBlockK, w.row0);
-          if (with_sf) bulk_load(sSF, sfa_src + static_cast<size_t>(kb >> 2) * kSfaBytes, kSfaBytes, full);
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
-        }
-      }
-    }
-  } else if (warp == 3) {
-    // ------------------------------- dependency scout -----------------------------------------
-    // Runs ahead through this CTA's down tiles: waits (bounded) until the four epilogue warp pairs of
-    // every gate/up tile of the tile's 128 rows have published their H rows, then tells the
-    // activation producer through s_dep.  The last down tile of an M-tile to get here puts the
-    // two global counters back to zero, so the workspace is clean when the kernel ends.
-    if (lane == 0 && fused) {
-      TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
-      int side, x, cleared = 0;
-      const int want = 4 * p.side[0].NT;
-      bool ok = true;
-      while (ok && it.next(side, x)) {
-        if (side == 0) continue;
-        const WorkItem w = decode_item(1, x, s_toff, s_cold, G, order2, stride);
-        const int tau = w.row0 >> 7;
-        unsigned long long t0 = 0;
-        for (uint32_t spin = 0; ld_acquire(p.ready + tau) < want; ++spin) {
-          if ((spin & 63u) == 63u) {
-            if (*s_abort) { ok = false; break; }
-            const unsigned long long now = global_timer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > wait_ns) { *s_abort = 1; ok = false; break; }
+          *s_dep = ++cleared;                      // tell the producer first, then do the bookkeeping
+          if (atomicAdd(p.done + tau, 1) == p.side[1].NT - 1) {
+            atomicExch(p.ready + tau, 0);
+            atomicExch(p.done + tau, 0);
           }
         }
-        if (!ok) break;
-        __threadfence_block();
-        *s_dep = ++cleared;                      // tell the producer first, then do the bookkeeping
-        if (atomicAdd(p.done + tau, 1) == p.side[1].NT - 1) {
-          atomicExch(p.ready + tau, 0);
-          atomicExch(p.done + tau, 0);
-        }
       }
-    }
-  } else if (warp == 1) {
-    // ------------------------------- MMA issuer -----------------------------------------------
-    if (lane == 0) {
-      uint32_t stage = 0, phase = 0, acc_phase = 0;
-      bool ok = true;
-      TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
-      int side, x;
-      while (ok && it.next(side, x)) {
-        const int Kb = p.side[side].Kb;
-        if (!mbar_wait(smem_u32(&s_acc_empty), acc_phase ^ 1u, s_abort, wait_ns)) break;
-        tc_fence_after();
-#pragma unroll 1
-        for (int kb = 0; kb < Kb; ++kb) {
-          if (!mbar_wait(smem_u32(&s_full[stage]), phase, s_abort, wait_ns)) { ok = false; break; }
+    } else if (warp == 1) {
+      // ------------------------------- MMA issuer -----------------------------------------------
+      if (lane == 0) {
+        uint32_t stage = 0, phase = 0, acc_phase = 0;
+        bool ok = true;
+        TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+        int side, x;
+        while (ok && it.next(side, x)) {
+          const int Kb = p.side[side].Kb;
+          if (!mbar_wait(smem_u32(&s_acc_empty), acc_phase ^ 1u, s_abort, wait_ns)) break;
           tc_fence_after();
-          const uint32_t sA = smem_base + stage * kStageBytes, sB = sA + kABytes, sSF = sB + kBBytes;
-          const uint32_t sfa_t = tmem_base + kSfCol0 + 16u * ((kb >> 2) & 1);
-          const uint32_t sfb_t = sfa_t + 4;
-          const uint64_t da = smem_desc_sw128(sA), db = smem_desc_sw128(sB);
-          if constexpr (kBf16) {
+#pragma unroll 1
+          for (int kb = 0; kb < Kb; ++kb) {
+            if (!mbar_wait(smem_u32(&s_full[stage]), phase, s_abort, wait_ns)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t sA = smem_base + stage * kStageBytes, sB = sA + kABytes, sSF = sB + kBBytes;
+            const uint32_t sfa_t = tmem_base + kSfCol0 + 16u * ((kb >> 2) & 1);
+            const uint32_t sfb_t = sfa_t + 4;
+            const uint64_t da = smem_desc_sw128(sA), db = smem_desc_sw128(sB);
+            if constexpr (kBf16) {
 #pragma unroll
-            for (int ks = 0; ks < kBlockK / 32; ++ks)     // 16 bf16 values = 32 bytes per instruction
-              tc_mma_bf16(tmem_base, da + 2u * ks, db + 2u * ks, instr_desc_bf16(), (kb | ks) != 0 ? 1u : 0u);
-          } else {
-            if ((kb & 3) == 0) {
-              tc_cp_sf(sfa_t, smem_desc_sf(sSF));
-              tc_cp_sf(sfb_t, smem_desc_sf(sSF + kSfaBytes));
-              tc_cp_sf(sfb_t + 4, smem_desc_sf(sSF + kSfaBytes + 512));
+              for (int ks = 0; ks < kBlockK / 32; ++ks)     // 16 bf16 values = 32 bytes per instruction
+                tc_mma_bf16(tmem_base, da + 2u * ks, db + 2u * ks, instr_desc_bf16(), (kb | ks) != 0 ? 1u : 0u);
+            } else {
+              if ((kb & 3) == 0) {
+                tc_cp_sf(sfa_t, smem_desc_sf(sSF));
+                tc_cp_sf(sfb_t, smem_desc_sf(sSF + kSfaBytes));
+                tc_cp_sf(sfb_t + 4, smem_desc_sf(sSF + kSfaBytes + 512));
+              }
+              const uint32_t idesc = instr_desc(kb & 3);
+#pragma unroll
+              for (int ks = 0; ks < kBlockK / 32; ++ks)
+                tc_mma_mxf8(tmem_base, da + 2u * ks, db + 2u * ks, idesc, sfa_t, sfb_t, (kb | ks) != 0 ? 1u : 0u);
             }
-            const uint32_t idesc = instr_desc(kb & 3);
-#pragma unroll
-            for (int ks = 0; ks < kBlockK / 32; ++ks)
-              tc_mma_mxf8(tmem_base, da + 2u * ks, db + 2u * ks, idesc, sfa_t, sfb_t, (kb | ks) != 0 ? 1u : 0u);
+            tc_commit(smem_u32(&s_empty[stage]));
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
           }
-          tc_commit(smem_u32(&s_empty[stage]));
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (ok) tc_commit(smem_u32(&s_acc_full));
+          acc_phase ^= 1u;
         }
-        if (ok) tc_commit(smem_u32(&s_acc_full));
-        acc_phase ^= 1u;
       }
     }
-  } else if (warp >= kEpiWarp0) {
+  } else if (kGather && warp >= kGatherWarp0) {
+    if constexpr (kGather) asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
+    // ------------------------------- row gather (gate/up operand) -------------------------------
+    // Warp gw owns rows gw*32 .. gw*32+31 of the A tile.  A lane copies one 16-byte chunk (lane & 7) of a
+    // row; the warp covers four rows per instruction (full 128-byte lines) and its 32 rows in eight.  A copy
+    // group is retired one K-block later: wait for it, make it visible to the tensor core's reads (async
+    // proxy), then one lane arrives on the stage's barrier - so copies of two stages are always in flight.
+    const int gw = warp - kGatherWarp0;
+    const int chunk = lane & 7, sub = lane >> 3;
+    const int kshift = (p.k & (p.k - 1)) == 0 ? __ffs(p.k) - 1 : -1;
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
+    int side, x;
+    while (ok && it.next(side, x)) {
+      const int Kb = p.side[side].Kb;
+      if (side == 1) {
+        const uint32_t adv = stage + static_cast<uint32_t>(Kb);
+        phase ^= (adv / kStages) & 1u;
+        stage = adv % kStages;
+        continue;
+      }
+      const WorkItem w = decode_item(0, x, s_toff, s_cold, G, order1, stride);
+      // byte offset of each of this lane's eight rows in x_q (-1: a row without a pair, zero-filled)
+      long long src_off[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int pr = __ldg(p.row_pair + w.row0 + gw * 32 + i * 4 + sub);
+        const int t = pr < 0 ? -1 : min(kshift >= 0 ? pr >> kshift : pr / p.k, p.T - 1);
+        src_off[i] = t < 0 ? -1 : static_cast<long long>(t) * p.d + chunk * 16;
+      }
+      const int pr_sf = __ldg(p.row_pair + w.row0 + gw * 32 + lane);       // this lane's row of the scale atom
+      const int t_sf = pr_sf < 0 ? -1 : min(kshift >= 0 ? pr_sf >> kshift : pr_sf / p.k, p.T - 1);
+      const uint8_t* sf_src = t_sf < 0 ? p.x_sf : p.x_sf + static_cast<size_t>(t_sf) * p.x_sf_stride;
+      int prev_stage = -1;
+#pragma unroll 1
+      for (int kb = 0; kb < Kb; ++kb) {
+        if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
+        const uint32_t sA = smem_base + stage * kStageBytes, sSF = sA + kABytes + kBBytes;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int r = gw * 32 + i * 4 + sub;
+          const uint32_t dst = sA + r * 128 + ((chunk ^ (r & 7)) << 4);
+          const bool live = src_off[i] >= 0;
+          cp_async_16(dst, p.x_q + (live ? src_off[i] + static_cast<long long>(kb) * kBlockK : 0), live ? 16u : 0u);
+        }
+        if ((kb & 3) == 0) cp_async_4(sSF + lane * 16 + gw * 4, sf_src + kb, t_sf >= 0 ? 4u : 0u);
+        cp_async_commit();
+        if (prev_stage >= 0) {
+          cp_async_wait<1>();
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&s_full[prev_stage]));
+        }
+        prev_stage = static_cast<int>(stage);
+        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+      }
+      cp_async_wait<0>();
+      if (prev_stage >= 0 && ok) {
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&s_full[prev_stage]));
+      }
+    }
+  } else {
+    if constexpr (kGather) asm volatile("setmaxnreg.inc.sync.aligned.u32 176;");
     // ------------------------------- epilogue --------------------------------------------------
     // Warps w and w + 4 read the same tensor-memory lane quadrant (rows quad*32 .. +31 of the tile)
     // and split each row's columns.  The accumulator is copied raw into registers and released
@@ -487,24 +574,30 @@ size_t ffn_workspace_bytes(int M_cap) {
   return ((2 * sizeof(int32_t) * static_cast<size_t>(M_cap / kTileM)) + 255) & ~static_cast<size_t>(255);
 }
 
-template <bool kBf16>
+template <bool kBf16, bool kGather>
 static cudaError_t launch_ffn_t(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
                                 const FfnParams& p, int num_sms, cudaStream_t stream) {
   static std::atomic<unsigned long long> smem_set{0};
-  cudaError_t e = smem_limit_once(ffn_kernel<kBf16>, kGemmSmemBytes, smem_set);
+  cudaError_t e = smem_limit_once(ffn_kernel<kBf16, kGather>, kGemmSmemBytes, smem_set);
   if (e != cudaSuccess) return e;
   const int grid = max(1, num_sms);   // one persistent CTA per SM; CTAs without work leave at once
-  return launch_pdl(ffn_kernel<kBf16>, dim3(grid), dim3(kGemmThreads), kGemmSmemBytes, stream, tmA1, tmA2, tmY, p);
+  return launch_pdl(ffn_kernel<kBf16, kGather>, dim3(grid), dim3(kGather ? kGatherThreads : kGemmThreads), kGemmSmemBytes,
+                    stream, tmA1, tmA2, tmY, p);
 }
 
 cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
                        const FfnParams& p, int num_sms, cudaStream_t stream) {
-  return launch_ffn_t<false>(tmA1, tmA2, tmY, p, num_sms, stream);
+  return launch_ffn_t<false, false>(tmA1, tmA2, tmY, p, num_sms, stream);
+}
+
+cudaError_t launch_ffn_gather(const CUtensorMap& tmA2, const CUtensorMap& tmY, const FfnParams& p, int num_sms,
+                              cudaStream_t stream) {
+  return launch_ffn_t<false, true>(tmA2, tmA2, tmY, p, num_sms, stream);   // the first map is never used
 }
 
 cudaError_t launch_ffn_bf16(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
                             const FfnParams& p, int num_sms, cudaStream_t stream) {
-  return launch_ffn_t<true>(tmA1, tmA2, tmY, p, num_sms, stream);
+  return launch_ffn_t<true, false>(tmA1, tmA2, tmY, p, num_sms, stream);
 }
 
 }  // namespace tempo

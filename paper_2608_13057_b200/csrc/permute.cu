@@ -258,6 +258,81 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_wave_kernel(const Per
   }
 }
 
+// Step 2 without the layout: quantise every live token row ONCE, in token order (x_q[t,:], one scale byte per
+// 128 columns in x_sf[t, :]), for the FFN entry point that gathers its rows itself (tempo_grouped_ffn_gather).
+// Nothing here depends on step 1, so the kernel does not wait for it at its start: launched behind the
+// dispatch kernel it runs beside it on the SMs the dispatch cluster leaves free.  It waits for its predecessor
+// only at its end, so that "this kernel is complete" still implies "step 1 is complete" for the kernel after it.
+// One warp per (token, 512-column chunk), two in flight, grid-stride.
+__global__ void __launch_bounds__(kPermWarps * 32) quantize_tokens_kernel(const QuantizeParams p) {
+  const int lane = threadIdx.x & 31;
+  const int chunks = (p.d + 511) >> 9;
+  int nv = p.T;
+  if (p.n_valid != nullptr) nv = max(0, min(*p.n_valid, p.T));     // an input of the step, not a result of step 1
+  const long long S = static_cast<long long>(gridDim.x) * kPermWarps;
+  const long long g0 = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5);
+  const long long n_items = static_cast<long long>(nv) * chunks;
+  for (long long g = g0; g < n_items; g += 2 * S) {
+    uint4 lo[2], hi[2];
+    int t[2], col[2];
+    bool in[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const long long gi = g + u * S;
+      const bool live = gi < n_items;
+      t[u] = live ? static_cast<int>(gi / chunks) : 0;
+      col[u] = live ? static_cast<int>(gi % chunks) * 512 + lane * 16 : 0;
+      in[u] = live && col[u] < p.d;
+      lo[u] = make_uint4(0, 0, 0, 0);
+      hi[u] = make_uint4(0, 0, 0, 0);
+      if (in[u]) {
+        const __nv_bfloat16* src = p.x + static_cast<size_t>(t[u]) * p.d + col[u];
+        lo[u] = __ldcs(reinterpret_cast<const uint4*>(src));
+        hi[u] = __ldcs(reinterpret_cast<const uint4*>(src + 8));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const uint32_t w[8] = {lo[u].x, lo[u].y, lo[u].z, lo[u].w, hi[u].x, hi[u].y, hi[u].z, hi[u].w};
+      __nv_bfloat162 m2 = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[0]));
+#pragma unroll
+      for (int i = 1; i < 8; ++i) m2 = __hmax2(m2, __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[i])));
+      const uint32_t mbits = *reinterpret_cast<const uint32_t*>(&m2);
+      float amax = fmaxf(__uint_as_float(mbits << 16), __uint_as_float(mbits & 0xffff0000u));
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
+      if (!in[u]) continue;
+      const int eps = pow2_scale_exponent(amax);
+      const float inv = pow2_neg(eps);
+      float v[16];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+      }
+      uint4 q;
+      q.x = cvt_e4m3x4(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv);
+      q.y = cvt_e4m3x4(v[4] * inv, v[5] * inv, v[6] * inv, v[7] * inv);
+      q.z = cvt_e4m3x4(v[8] * inv, v[9] * inv, v[10] * inv, v[11] * inv);
+      q.w = cvt_e4m3x4(v[12] * inv, v[13] * inv, v[14] * inv, v[15] * inv);
+      *reinterpret_cast<uint4*>(p.x_q + static_cast<size_t>(t[u]) * p.d + col[u]) = q;     // re-read soon: keep it in L2
+      if ((lane & 7) == 0) p.x_sf[static_cast<size_t>(t[u]) * p.sf_stride + (col[u] >> 7)] = static_cast<uint8_t>(eps + 127);
+    }
+  }
+  pdl_wait();
+  pdl_trigger();
+}
+
+cudaError_t launch_quantize_tokens(const QuantizeParams& p, int num_sms, cudaStream_t stream) {
+  const long long warps = static_cast<long long>(p.T) * ((p.d + 511) >> 9);
+  long long blocks = (warps + 2 * kPermWarps - 1) / (2 * kPermWarps);
+  const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 6;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return launch_pdl(quantize_tokens_kernel, dim3(static_cast<unsigned int>(blocks)), dim3(kPermWarps * 32), 0, stream, p);
+}
+
 // bf16 variant of step 2: the gathered rows stay bf16 (no quantiser); rows without a pair are zero.
 // One warp per (row, 512-byte chunk), 16 bytes per lane.
 __global__ void __launch_bounds__(kPermWarps * 32) permute_pad_bf16_kernel(const PermuteParams p, __nv_bfloat16* a) {

@@ -62,6 +62,16 @@ struct PermuteParams {
 cudaError_t launch_permute_pad(const PermuteParams& p, int num_sms, cudaStream_t stream);
 cudaError_t launch_permute_pad_bf16(const PermuteParams& p, __nv_bfloat16* a, int num_sms, cudaStream_t stream);
 
+struct QuantizeParams {
+  int T, d;
+  int sf_stride;              // bytes per token of x_sf: 4 * ceil((d / 128) / 4)
+  const __nv_bfloat16* x;
+  const int32_t* n_valid;
+  uint8_t* x_q;
+  uint8_t* x_sf;
+};
+cudaError_t launch_quantize_tokens(const QuantizeParams& p, int num_sms, cudaStream_t stream);
+
 struct CombineParams {
   int T, k, d;
   const __nv_bfloat16* y;
@@ -108,6 +118,11 @@ struct FfnParams {
   uint8_t* h_q;
   uint8_t* h_sf;
   __nv_bfloat16* y;
+  // gather form (ffn_kernel<false, true>): the gate/up operand rows are fetched from the per-token buffers
+  const uint8_t* x_q;        // e4m3 codes [T, d]
+  const uint8_t* x_sf;       // scale bytes [T, x_sf_stride]
+  const int32_t* row_pair;   // row -> pair (token = pair / k), -1: zero row
+  int x_sf_stride, k, T;
   int32_t* ready;        // workspace: per M-tile, epilogue warps of finished gate/up tiles
   int32_t* done;         // workspace: per M-tile, down tiles that have seen `ready` complete
   uint32_t* status;
@@ -119,6 +134,8 @@ cudaError_t launch_ffn_bf16(const CUtensorMap& tmA1, const CUtensorMap& tmA2, co
                             const FfnParams& p, int num_sms, cudaStream_t stream);
 cudaError_t launch_ffn(const CUtensorMap& tmA1, const CUtensorMap& tmA2, const CUtensorMap& tmY,
                        const FfnParams& p, int num_sms, cudaStream_t stream);
+cudaError_t launch_ffn_gather(const CUtensorMap& tmA2, const CUtensorMap& tmY, const FfnParams& p, int num_sms,
+                              cudaStream_t stream);
 
 
 }  // namespace tempo
