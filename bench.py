@@ -627,7 +627,7 @@ def run_gpu(args):
 
     K, Wm, R = args.steps, args.warmup, max(1, args.replays)
     wl = make_workload(args.workload, rank)
-    leg = Leg(torch, B, args.workload, wl, max_m=args.max_m, path=args.path)
+    leg = Leg(torch, B, args.workload, wl, max_m=args.max_m, path=args.path, device_weights=args.device_weights)
     st = leg.st
     sampler = ClockSampler(local) if rank == 0 else None
 
@@ -711,7 +711,7 @@ def run_gpu(args):
                       **{k: {kk: fit[k][kk] for kk in keep} for k in ("fit_ffn", "fit_ffn_tile", "fit_block", "fit_block_tile")},
                       "points": [{k: r[k] for k in ("G", "n", "t_ffn_us", "t_block_us")} for r in fit["rows"]]}
         out["measured_fp8"] = fp8
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and not args.device_weights:
         v, sample = oracle_sample_us_per_block(wl, budget_s=12.0)
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle", "sample": sample}
     print(json.dumps(out))
@@ -754,6 +754,8 @@ def main():
     ap.add_argument("--path", default="permute", choices=["permute", "gather"],
                     help="steps 2-3: tempo_permute_pad + tempo_grouped_ffn, or tempo_quantize_tokens + "
                          "tempo_grouped_ffn_gather (same results bit for bit)")
+    ap.add_argument("--device-weights", action="store_true",
+                    help="draw the weights on the device (timing only; minutes faster for the large shapes)")
     ap.add_argument("--max-m", type=int, default=0, help="> 0: run the block in the masked layout with this row stride")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -8,7 +8,7 @@ namespace tempo {
 constexpr int kDispThreads = 1024;
 constexpr int kDispWarps = kDispThreads / 32;
 constexpr int kKeep = 4;           // 32-pair steps of a warp whose ids stay in registers between the passes
-constexpr int kMaxCluster = 8;     // portable cluster size
+constexpr int kMaxCluster = 16;    // largest cluster on this part (beyond 8 is opt-in per kernel; checked per device)
 constexpr int kPairsPerCta = 1024;
 constexpr int kMaxShare = 1 << 30;   // largest share x_{e,r} the quota dispatch accepts
 constexpr size_t kDispatchSmemLimit = 220 * 1024;   // the shape check rejects tables beyond this // pairs per CTA before another CTA joins the cluster
@@ -56,10 +56,42 @@ __device__ __forceinline__ int instance_of_row(const int32_t* off, int G, int ro
   return lo;
 }
 
-inline int dispatch_cluster_size(long long pairs) {
+inline int dispatch_cluster_size(long long pairs, int max_cluster) {
   int nc = 1;
-  while (nc < kMaxCluster && static_cast<long long>(nc) * kPairsPerCta < pairs) nc *= 2;
+  while (nc < max_cluster && static_cast<long long>(nc) * kPairsPerCta < pairs) nc *= 2;
   return nc;
+}
+
+// Largest cluster the kernel can run on the current device: 16 where the device can place a cluster of 16
+// such CTAs in one GPC (asked once per device), else the portable 8.
+template <typename Params>
+inline int dispatch_max_cluster(void (*kernel)(Params), size_t smem) {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 8;
+  const int have = cached[dev].load(std::memory_order_acquire);
+  if (have != 0) return have;
+  int best = 8;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kMaxCluster);
+    cfg.blockDim = dim3(kDispThreads);
+    cfg.dynamicSmemBytes = smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kMaxCluster;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) == cudaSuccess && n > 0) best = kMaxCluster;
+    else (void)cudaGetLastError();                 // a refused query must not poison the next launch
+  } else {
+    (void)cudaGetLastError();
+  }
+  cached[dev].store(best, std::memory_order_release);
+  return best;
 }
 
 template <typename Params>
@@ -69,7 +101,7 @@ inline cudaError_t launch_dispatch_cluster(void (*kernel)(Params), const Params&
   static std::atomic<unsigned long long> smem_set{0};
   cudaError_t e = smem_limit_once(kernel, kDispatchSmemLimit, smem_set);
   if (e != cudaSuccess) return e;
-  const int nc = dispatch_cluster_size(pairs);
+  const int nc = dispatch_cluster_size(pairs, dispatch_max_cluster(kernel, kDispatchSmemLimit));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(nc);
   cfg.blockDim = dim3(kDispThreads);

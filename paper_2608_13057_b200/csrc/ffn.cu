@@ -197,10 +197,15 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
           const WorkItem w = decode_item(side, x, s_toff, s_cold, G, side == 0 ? order1 : order2, stride);
           const uint8_t* sfa_src = gs.sfa + static_cast<size_t>(w.row0 >> 7) * gs.JK * kSfaBytes;
           const CUtensorMap* tm = side == 0 ? &tmA1 : &tmA2;
-          if (kGather && side == 0) {                      // the gather warps fill these stages
-            const uint32_t adv = stage + static_cast<uint32_t>(gs.Kb);
-            phase ^= (adv / kStages) & 1u;
-            stage = adv % kStages;
+          if (kGather && side == 0) {
+            // The gather warps fill these stages.  This thread still follows the ring slot by slot: an
+            // mbarrier wait tells one phase from the next only, so a waiter that jumped several phases
+            // ahead would take a stage that is still in use for a free one.
+#pragma unroll 1
+            for (int kb = 0; kb < gs.Kb; ++kb) {
+              if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
+              if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
             continue;
           }
           if (side == 1 && fused) {
@@ -327,10 +332,12 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
     int side, x;
     while (ok && it.next(side, x)) {
       const int Kb = p.side[side].Kb;
-      if (side == 1) {
-        const uint32_t adv = stage + static_cast<uint32_t>(Kb);
-        phase ^= (adv / kStages) & 1u;
-        stage = adv % kStages;
+      if (side == 1) {                                   // follow the ring slot by slot (see the activation producer)
+#pragma unroll 1
+        for (int kb = 0; kb < Kb; ++kb) {
+          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
         continue;
       }
       const WorkItem w = decode_item(0, x, s_toff, s_cold, G, order1, stride);

@@ -34,6 +34,7 @@ def _cases():
     yield W.random_small(400, T=40, E=6, k=2, d=256, f=384)
     yield W.random_small(410, T=40, n_valid=23)
     yield W.random_small(411, T=50, E=7, k=3, R_max=3, n_valid=41)   # k not a power of two
+    yield W.config5_point(48, 130, d=256, f=512)          # 480 tiles: every CTA takes several, gate/up then down
     yield W.config2()
     yield W.config2(n_valid=200)
 
