@@ -736,6 +736,68 @@ def run_sweep(args):
     print(json.dumps(result))
 
 
+# --------------------------------------------------------------------------------------------------
+# dispatch policies on the mixed-regime batch: modelled against measured (closes the solver loop)
+# --------------------------------------------------------------------------------------------------
+
+def run_policies(args):
+    """Config 3's routed batch under four dispatch policies (uniform, token-balanced, keep-hot-whole, and the
+    table tempo_fast builds from the cost profile fitted IN THIS RUN): for each, the block time of the rank
+    that holds all 20 slots and of the two virtual GPUs (16 primaries / 4 replica slots) the solver balances,
+    measured on this GPU one after the other, next to what the fitted Eq. 3 profile predicts."""
+    import torch
+    from paper_2608_13057_b200 import binding as B
+    from paper_2608_13057_b200 import policies as P
+    from paper_2608_13057_b200 import solver as S
+
+    torch.cuda.set_device(0)
+
+    def barrier():
+        torch.cuda.synchronize()
+
+    if args.fit_json:
+        fit = json.load(open(args.fit_json))
+        fit = fit.get("fit", fit)["fit_block_tile"]
+    else:
+        rows = sweep_rows(torch, B, FIT_G, FIT_N, max(10, min(args.replays, 30)), device_weights=True)
+        fit = fit_rows(rows)["fit_block_tile"]
+    params = S.CostParams(a=fit["a"], b=fit["b"], c=fit["c"], beta=fit["beta"], b2=fit["b2"])
+    K, R = args.steps, max(1, args.replays)
+    out = {"policies": [], "fit_block_tile": {k: fit[k] for k in ("a", "b", "b2", "c", "beta", "n_star", "fit_err")},
+           "workload": "cfg3 routed batch (T=4096, top-8, Zipf 1.2), 16 primaries on virtual GPU A, replicas of the "
+                       "4 hottest on virtual GPU B", "steps_per_region": K, "regions": R}
+    for case in P.build_cases(params):
+        m = P.modeled(case.x, params)
+        meas = {}
+        for key, wl in (("rank", case.rank), ("gpu_a", case.gpus[0]), ("gpu_b", case.gpus[1])):
+            leg = Leg(torch, B, wl.name, wl, device_weights=True, path=args.path)
+            ms = leg.time_regions(K, 3, R, barrier)
+            status = int(leg.buf.status.item())
+            # the quota table is honoured exactly: every instance holds the rows the policy gave it
+            want = np.zeros(wl.G_max, np.int64)
+            for e in range(wl.E):
+                for r in range(wl.R_max):
+                    if wl.replica_map[e, r] >= 0:
+                        want[wl.replica_map[e, r]] = wl.quota[e, r]
+            exact = bool(np.array_equal(leg.buf.inst_count.cpu().numpy(), want))
+            meas[key] = dict(us=float(np.median(ms)) / K * 1e3, status=status, quotas_exact=exact, G_act=leg.st["G_act"],
+                             N=leg.st["N_local"], tiles=leg.st["tiles"])
+            del leg
+            torch.cuda.empty_cache()
+        hot = [[int(a), int(b)] for a, b in case.x if b > 0]
+        out["policies"].append(dict(policy=case.name, hot_splits=hot, modeled_us=m,
+                                    measured_us=dict(gpu_us=[meas["gpu_a"]["us"], meas["gpu_b"]["us"]],
+                                                     makespan_us=max(meas["gpu_a"]["us"], meas["gpu_b"]["us"]),
+                                                     rank_us=meas["rank"]["us"]),
+                                    detail=meas))
+    mk = [p["measured_us"]["makespan_us"] for p in out["policies"]]
+    md = [p["modeled_us"]["makespan_us"] for p in out["policies"]]
+    out["spread"] = {"measured_worst_over_best": max(mk) / min(mk), "modeled_worst_over_best": max(md) / min(md),
+                     "measured_best": out["policies"][int(np.argmin(mk))]["policy"],
+                     "modeled_best": out["policies"][int(np.argmin(md))]["policy"]}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -747,6 +809,9 @@ def main():
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the linear-regime leg, the in-run fit and the fp8 GEMM rate of the default line")
     ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--policies", action="store_true",
+                    help="config 3 under four dispatch policies: modelled (fit of this run) against measured")
+    ap.add_argument("--fit-json", default="", help="--policies: take fit_block_tile from this bench line instead")
     ap.add_argument("--sweep-G", default="")
     ap.add_argument("--sweep-N", default="")
     ap.add_argument("--replays", type=int, default=30, help="timed regions of K steps each (sweep: replays per point)")
@@ -763,6 +828,8 @@ def main():
         run_reference(args)
     elif args.sweep:
         run_sweep(args)
+    elif args.policies:
+        run_policies(args)
     else:
         run_gpu(args)
 

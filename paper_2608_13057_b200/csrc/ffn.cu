@@ -54,10 +54,10 @@ constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 4
 // (12-15) fetch each row of the A tile from the per-token quantised activations x_q by the row's
 // token (row_pair / k) with 16-byte cp.async copies straight into the 128-byte-swizzled stage, and its
 // scale bytes from x_sf into the stage's scale atom; rows without a pair are zero-filled.  That takes
-// the permuted a_q / a_sf buffers (one write and NT re-reads of every row) out of the block.  The
-// stage's "full" barrier then counts five arrivals (weights + four gather warps) instead of two; on
-// down tiles the activation producer makes up the difference.  512 threads leave 128 registers per
-// thread at launch; the producer and gather warps hand most of theirs to the epilogue warps (setmaxnreg).
+// the permuted a_q / a_sf buffers (one write and NT re-reads of every row) out of the block.  Each
+// gather warp owns one stage of the ring and is that stage's second arrival on gate/up tiles, as the
+// activation producer is on down tiles.  512 threads leave 128 registers per thread at launch; the
+// producer and gather warps hand most of theirs to the epilogue warps (setmaxnreg).
 template <bool kBf16, bool kGather>
 __global__ void __launch_bounds__(kGather ? kGatherThreads : kGemmThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
@@ -84,7 +84,7 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   pdl_trigger();
   // prologue that needs nothing from the previous kernel: barriers, tensor memory, descriptor fetch
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), kGather ? 5 : 2); mbar_init(smem_u32(&s_empty[s]), 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(smem_u32(&s_full[s]), 2); mbar_init(smem_u32(&s_empty[s]), 1); }
     mbar_init(smem_u32(&s_acc_full), 1);
     mbar_init(smem_u32(&s_acc_empty), 8);
     s_abort_storage = 0;
@@ -234,7 +234,6 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
             const uint32_t sA = smem_base + stage * kStageBytes, sSF = sA + kABytes + kBBytes;
             const bool with_sf = !kBf16 && (kb & 3) == 0;
             mbar_arrive_expect_tx(full, kABytes + (with_sf ? kSfaBytes : 0));
-            if constexpr (kGather) mbar_arrive_n(full, 3);   // stands in for the gather warps, idle on down tiles
             tma_load_2d(sA, tm, full, kb * kBlockK, w.row0);
             if (with_sf) bulk_load(sSF, sfa_src + static_cast<size_t>(kb >> 2) * kSfaBytes, kSfaBytes, full);
             if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -319,67 +318,78 @@ ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUt
   } else if (kGather && warp >= kGatherWarp0) {
     if constexpr (kGather) asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
     // ------------------------------- row gather (gate/up operand) -------------------------------
-    // Warp gw owns rows gw*32 .. gw*32+31 of the A tile.  A lane copies one 16-byte chunk (lane & 7) of a
-    // row; the warp covers four rows per instruction (full 128-byte lines) and its 32 rows in eight.  A copy
-    // group is retired one K-block later: wait for it, make it visible to the tensor core's reads (async
-    // proxy), then one lane arrives on the stage's barrier - so copies of two stages are always in flight.
+    // Each of the four warps owns ONE stage of the ring (warp gw takes every K-block that lands in stage gw)
+    // and copies all 128 rows of its K-block: a lane copies the 16-byte chunk (lane & 7) of 32 rows, so one
+    // instruction of the warp covers four whole 128-byte rows.  It then waits for its own copies, makes them
+    // visible to the tensor core's reads (async proxy) and arrives on the stage's barrier; meanwhile the other
+    // three warps have their K-blocks in flight, so four stages of activations are under way at once, as
+    // with the tensor copies of the permuted form.  On down tiles the warp only follows its stage's phases:
+    // an mbarrier wait tells one phase from the next only, so nobody may skip ahead.
+    static_assert(kStages == 4, "one gather warp per stage");
     const int gw = warp - kGatherWarp0;
     const int chunk = lane & 7, sub = lane >> 3;
     const int kshift = (p.k & (p.k - 1)) == 0 ? __ffs(p.k) - 1 : -1;
-    uint32_t stage = 0, phase = 0;
+    const uint32_t d16 = static_cast<uint32_t>(p.d) >> 4;          // row pitch of x_q in 16-byte units
+    const uint4* xq16 = reinterpret_cast<const uint4*>(p.x_q);
+    const uint32_t my_empty = smem_u32(&s_empty[gw]), my_full = smem_u32(&s_full[gw]);
+    const uint32_t sA = smem_base + gw * kStageBytes, sSF = sA + kABytes + kBBytes;
+    uint32_t phase = 0;
+    uint32_t cnt = 0;                                              // K-blocks of this CTA so far (stage = cnt % 4)
     bool ok = true;
     TileIter it(blockIdx.x, gridDim.x, n1, n2, Kb1, Kb2);
     int side, x;
     while (ok && it.next(side, x)) {
       const int Kb = p.side[side].Kb;
-      if (side == 1) {                                   // follow the ring slot by slot (see the activation producer)
+      // first K-block of this tile in my stage, and how many of them
+      int kb = static_cast<int>((static_cast<uint32_t>(gw) - cnt) & (kStages - 1));
+      cnt += static_cast<uint32_t>(Kb);
+      if (side == 1) {
 #pragma unroll 1
-        for (int kb = 0; kb < Kb; ++kb) {
-          if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        for (; kb < Kb; kb += kStages) {
+          if (!mbar_wait(my_empty, phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
+          phase ^= 1u;
         }
         continue;
       }
       const WorkItem w = decode_item(0, x, s_toff, s_cold, G, order1, stride);
-      // byte offset of each of this lane's eight rows in x_q (-1: a row without a pair, zero-filled)
-      long long src_off[8];
+      // x_q offset (16-byte units) of each of this lane's 32 rows; ~0: a row without a pair, zero-filled
+      uint32_t off16[32];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int pr = __ldg(p.row_pair + w.row0 + gw * 32 + i * 4 + sub);
-        const int t = pr < 0 ? -1 : min(kshift >= 0 ? pr >> kshift : pr / p.k, p.T - 1);
-        src_off[i] = t < 0 ? -1 : static_cast<long long>(t) * p.d + chunk * 16;
+      for (int i = 0; i < 32; ++i) {
+        const int pr = __ldg(p.row_pair + w.row0 + i * 4 + sub);
+        const int t = min(kshift >= 0 ? pr >> kshift : pr / p.k, p.T - 1);
+        off16[i] = pr < 0 ? 0xffffffffu : static_cast<uint32_t>(t) * d16 + chunk;
       }
-      const int pr_sf = __ldg(p.row_pair + w.row0 + gw * 32 + lane);       // this lane's row of the scale atom
-      const int t_sf = pr_sf < 0 ? -1 : min(kshift >= 0 ? pr_sf >> kshift : pr_sf / p.k, p.T - 1);
-      const uint8_t* sf_src = t_sf < 0 ? p.x_sf : p.x_sf + static_cast<size_t>(t_sf) * p.x_sf_stride;
-      int prev_stage = -1;
+      // scale atom: this lane supplies the 4-byte word of rows lane, lane + 32, lane + 64, lane + 96
+      int t_sf[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int pr = __ldg(p.row_pair + w.row0 + q * 32 + lane);
+        t_sf[q] = pr < 0 ? -1 : min(kshift >= 0 ? pr >> kshift : pr / p.k, p.T - 1);
+      }
 #pragma unroll 1
-      for (int kb = 0; kb < Kb; ++kb) {
-        if (!mbar_wait(smem_u32(&s_empty[stage]), phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
-        const uint32_t sA = smem_base + stage * kStageBytes, sSF = sA + kABytes + kBBytes;
+      for (; kb < Kb; kb += kStages) {
+        if (!mbar_wait(my_empty, phase ^ 1u, s_abort, wait_ns)) { ok = false; break; }
+        phase ^= 1u;
+        const uint32_t kb16 = static_cast<uint32_t>(kb) * (kBlockK / 16);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int r = gw * 32 + i * 4 + sub;
+        for (int i = 0; i < 32; ++i) {
+          const int r = i * 4 + sub;
           const uint32_t dst = sA + r * 128 + ((chunk ^ (r & 7)) << 4);
-          const bool live = src_off[i] >= 0;
-          cp_async_16(dst, p.x_q + (live ? src_off[i] + static_cast<long long>(kb) * kBlockK : 0), live ? 16u : 0u);
+          const bool live = off16[i] != 0xffffffffu;
+          cp_async_16(dst, xq16 + (live ? off16[i] + kb16 : 0u), live ? 16u : 0u);
         }
-        if ((kb & 3) == 0) cp_async_4(sSF + lane * 16 + gw * 4, sf_src + kb, t_sf >= 0 ? 4u : 0u);
+        if ((kb & 3) == 0) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            cp_async_4(sSF + lane * 16 + q * 4,
+                       p.x_sf + (t_sf[q] < 0 ? 0 : static_cast<size_t>(t_sf[q]) * p.x_sf_stride + kb), t_sf[q] < 0 ? 0u : 4u);
+        }
         cp_async_commit();
-        if (prev_stage >= 0) {
-          cp_async_wait<1>();
-          fence_async_smem();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&s_full[prev_stage]));
-        }
-        prev_stage = static_cast<int>(stage);
-        if (++stage == kStages) { stage = 0; phase ^= 1u; }
-      }
-      cp_async_wait<0>();
-      if (prev_stage >= 0 && ok) {
+        cp_async_wait<0>();
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&s_full[prev_stage]));
+        if (lane == 0) mbar_arrive(my_full);
       }
     }
   } else {

@@ -263,7 +263,9 @@ __global__ void __launch_bounds__(kPermWarps * 32) permute_wave_kernel(const Per
 // Nothing here depends on step 1, so the kernel does not wait for it at its start: launched behind the
 // dispatch kernel it runs beside it on the SMs the dispatch cluster leaves free.  It waits for its predecessor
 // only at its end, so that "this kernel is complete" still implies "step 1 is complete" for the kernel after it.
-// One warp per (token, 512-column chunk), two in flight, grid-stride.
+// One warp per (token, 512-column chunk), four in flight, grid-stride.
+constexpr int kQuantInFlight = 4;
+
 __global__ void __launch_bounds__(kPermWarps * 32) quantize_tokens_kernel(const QuantizeParams p) {
   const int lane = threadIdx.x & 31;
   const int chunks = (p.d + 511) >> 9;
@@ -272,12 +274,12 @@ __global__ void __launch_bounds__(kPermWarps * 32) quantize_tokens_kernel(const 
   const long long S = static_cast<long long>(gridDim.x) * kPermWarps;
   const long long g0 = static_cast<long long>(blockIdx.x) * kPermWarps + (threadIdx.x >> 5);
   const long long n_items = static_cast<long long>(nv) * chunks;
-  for (long long g = g0; g < n_items; g += 2 * S) {
-    uint4 lo[2], hi[2];
-    int t[2], col[2];
-    bool in[2];
+  for (long long g = g0; g < n_items; g += kQuantInFlight * S) {
+    uint4 lo[kQuantInFlight], hi[kQuantInFlight];
+    int t[kQuantInFlight], col[kQuantInFlight];
+    bool in[kQuantInFlight];
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < kQuantInFlight; ++u) {
       const long long gi = g + u * S;
       const bool live = gi < n_items;
       t[u] = live ? static_cast<int>(gi / chunks) : 0;
@@ -292,7 +294,7 @@ __global__ void __launch_bounds__(kPermWarps * 32) quantize_tokens_kernel(const 
       }
     }
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < kQuantInFlight; ++u) {
       const uint32_t w[8] = {lo[u].x, lo[u].y, lo[u].z, lo[u].w, hi[u].x, hi[u].y, hi[u].z, hi[u].w};
       __nv_bfloat162 m2 = __habs2(*reinterpret_cast<const __nv_bfloat162*>(&w[0]));
 #pragma unroll
@@ -326,7 +328,7 @@ __global__ void __launch_bounds__(kPermWarps * 32) quantize_tokens_kernel(const 
 
 cudaError_t launch_quantize_tokens(const QuantizeParams& p, int num_sms, cudaStream_t stream) {
   const long long warps = static_cast<long long>(p.T) * ((p.d + 511) >> 9);
-  long long blocks = (warps + 2 * kPermWarps - 1) / (2 * kPermWarps);
+  long long blocks = (warps + kQuantInFlight * kPermWarps - 1) / (kQuantInFlight * kPermWarps);
   const long long cap = static_cast<long long>(num_sms > 0 ? num_sms : 148) * 6;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;

@@ -613,3 +613,22 @@ def test_pack_rejects_non_power_of_two_scales(B):
     w2_s[0, 0, 0] = 0.3
     buf.pack_weights(w13_q, w13_s, w2_q, w2_s)
     assert int(buf.status.item()) & B.STATUS_BAD_SCALE
+
+
+def test_solver_table_reaches_the_dispatch_kernel_and_is_honoured_exactly(B):
+    """The off-path solver's output is the table the in-graph kernel reads (Section 4.2 -> Section 4.4): every
+    policy of the mixed-regime batch, the solver's included, goes through tempo_count_dispatch with status 0,
+    bit-exact against the oracle, every instance holding exactly the rows its share says."""
+    from paper_2608_13057_b200 import policies as P
+    from paper_2608_13057_b200 import solver as S
+    params = S.CostParams(a=28.4, b=3.42, c=-190.0, beta=0.0246, b2=2.31)       # a fitted B200 block-scope profile
+    for case in P.build_cases(params, with_x=False):
+        for wl in [case.rank] + case.gpus:
+            buf, got = _dispatch_only(B, wl)
+            ref = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, buf.M_cap)
+            _assert_dispatch_equal(got, ref)
+            assert got["status"] == 0
+            for e in range(wl.E):
+                for r in range(wl.R_max):
+                    if wl.replica_map[e, r] >= 0:
+                        assert int(got["inst_count"][wl.replica_map[e, r]]) == int(wl.quota[e, r])
