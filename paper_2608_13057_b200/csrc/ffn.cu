@@ -42,7 +42,7 @@ constexpr int kStages = 4;
 constexpr int kStageBytes = kABytes + kBBytes + 2048;     // 51200, a multiple of 1024
 constexpr int kGemmThreads = 384;
 constexpr int kEpiWarp0 = 4;                               // first of the 8 epilogue warps
-constexpr int kGatherWarp0 = 12;                           // gather form: 4 more warps, one per 32 rows of the A tile
+constexpr int kGatherWarp0 = 12;                           // gather form: 4 more warps, one per stage of the ring
 constexpr int kGatherThreads = 512;
 constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 4 * kStoreBytes + 1024;
 
@@ -57,7 +57,10 @@ constexpr size_t kGemmSmemBytes = static_cast<size_t>(kStages) * kStageBytes + 4
 // the permuted a_q / a_sf buffers (one write and NT re-reads of every row) out of the block.  Each
 // gather warp owns one stage of the ring and is that stage's second arrival on gate/up tiles, as the
 // activation producer is on down tiles.  512 threads leave 128 registers per thread at launch; the
-// producer and gather warps hand most of theirs to the epilogue warps (setmaxnreg).
+// producer and gather warps hand most of theirs to the epilogue warps (setmaxnreg).  Measured on B200 this
+// form's kernel is 15-25 % slower than the permuted form's (the tensor pipe waits for A rows that 16-byte
+// copies deliver later than one bulk tensor copy would): it is for callers who want the memory of the
+// permuted copy back, not for speed.
 template <bool kBf16, bool kGather>
 __global__ void __launch_bounds__(kGather ? kGatherThreads : kGemmThreads, 1)
 ffn_kernel(const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmA2,
