@@ -736,7 +736,7 @@ def run_gpu(args):
         "block_us": us_step, "block_us_percentiles": pct, "tokens_per_s": st["n_valid"] * world / (us_step * 1e-6),
         "block_roofline": block, "kernel_us": kern_us, "gpu_launches": 4 * K, "device_status": status,
         "roofline": roof, "clocks": clocks,
-        "e2e": {"value": ms_e2e_max * 1e3 / units, "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
+        "e2e": {"value": None if math.isnan(ms_e2e_max) else ms_e2e_max * 1e3 / units, "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
                 "d2h_bytes_per_step": e2e["d2h"], "pipeline": e2e["mode"], "steps": e2e["steps"],
                 "results_identical": e2e["identical"]},
     }
