@@ -796,8 +796,9 @@ def run_sweep(args):
 # --------------------------------------------------------------------------------------------------
 
 def run_policies(args):
-    """Config 3's routed batch under four dispatch policies (uniform, token-balanced, keep-hot-whole, and the
-    table tempo_fast builds from the cost profile fitted IN THIS RUN): for each, the block time of the rank
+    """Config 3's routed batch under five dispatch policies (uniform, token-balanced, keep-hot-whole, the table
+    tempo_fast builds from the cost profile fitted IN THIS RUN, and the same solved on the previous window's counts
+    as the deployed system does): for each, the block time of the rank
     that holds all 20 slots and of the two virtual GPUs (16 primaries / 4 replica slots) the solver balances,
     measured on this GPU one after the other, next to what the fitted Eq. 3 profile predicts."""
     import torch
@@ -830,10 +831,12 @@ def run_policies(args):
             status = int(leg.buf.status.item())
             # the quota table is honoured exactly: every instance holds the rows the policy gave it
             want = np.zeros(wl.G_max, np.int64)
-            for e in range(wl.E):
-                for r in range(wl.R_max):
-                    if wl.replica_map[e, r] >= 0:
-                        want[wl.replica_map[e, r]] = wl.quota[e, r]
+            if key == "rank":
+                want[:] = case.rank_rows                # what the (renormalised, if stale) table must give
+            else:
+                for e in range(wl.E):
+                    if wl.replica_map[e, 0] >= 0:
+                        want[wl.replica_map[e, 0]] = wl.quota[e, 0]
             exact = bool(np.array_equal(leg.buf.inst_count.cpu().numpy(), want))
             meas[key] = dict(us=float(np.median(ms)) / K * 1e3, status=status, quotas_exact=exact, G_act=leg.st["G_act"],
                              N=leg.st["N_local"], tiles=leg.st["tiles"])

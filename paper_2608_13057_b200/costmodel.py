@@ -16,6 +16,16 @@ from typing import Dict, Optional, Sequence
 import numpy as np
 
 
+def window_counts(cum_now, cum_prev) -> np.ndarray:
+    """Per-expert counts of the window between two snapshots of the cumulative u32 counter that
+    tempo_count_dispatch keeps (Section 4.4: cumulative counting needs no zeroing kernel in the graph; the
+    background thread recovers windows by wrap-safe differencing).  Exact as long as fewer than 2^32 pairs of
+    one expert fall into a window."""
+    now = np.asarray(cum_now).astype(np.uint32, copy=False)
+    prev = np.asarray(cum_prev).astype(np.uint32, copy=False)
+    return (now - prev).astype(np.uint32)          # unsigned subtraction wraps mod 2^32
+
+
 def tiles_of(rows: Sequence[int], tile: int = 128) -> int:
     return int(sum(-(-int(m) // tile) for m in rows if m > 0))
 

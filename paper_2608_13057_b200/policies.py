@@ -21,24 +21,43 @@ from typing import Dict, List, Sequence
 
 import numpy as np
 
+from . import costmodel as C
 from . import solver as S
 from . import workloads as W
 
-POLICIES = ("uniform", "token_balanced", "hot_whole", "tempo_fast")
+# tempo_fast_stale1 is the deployment the paper describes (Section 4.4, "Pricing staleness"): the table is solved on
+# the PREVIOUS window's counts, recovered from the cumulative counter, and the kernel renormalises its rows at use.
+POLICIES = ("uniform", "token_balanced", "hot_whole", "tempo_fast", "tempo_fast_stale1")
 
 
 @dataclasses.dataclass
 class PolicyCase:
     name: str
     x: np.ndarray                 # [n_local, 2] rows of each local expert on virtual GPU A / B
-    rank: W.Workload              # the rank holding all 20 slots, quota table from x
+    rank: W.Workload              # the rank holding all 20 slots, its quota table = the policy's (possibly stale) table
     gpus: List[W.Workload]        # [A, B]: the routed batch each virtual GPU sees, its own slots only
+    rank_rows: np.ndarray         # [20] rows every instance slot of the rank must end up with (x in slot order)
 
 
 def _local_counts(wl: W.Workload, local: Sequence[int]) -> List[int]:
     live = wl.topk_ids[:wl.n_valid].reshape(-1)
     c = np.bincount(live, minlength=wl.E)
     return [int(c[e]) for e in local]
+
+
+def renormalised(quota_row: Sequence[int], n_e: int) -> List[int]:
+    """Rows each replica column receives when a (possibly stale) share row meets n_e pairs: column r takes the
+    ranks [floor(C_{r-1} n_e / S), floor(C_r n_e / S)) with C the running sum of the shares, uniform if S = 0."""
+    q = [max(int(v), 0) for v in quota_row]
+    if sum(q) == 0:
+        q = [1] * len(q)
+    S_, out, C_, prev = sum(q), [], 0, 0
+    for v in q:
+        C_ += v
+        b = (C_ * int(n_e)) // S_
+        out.append(b - prev)
+        prev = b
+    return out
 
 
 def shares(policy: str, counts: Sequence[int], hot: Sequence[int], params: S.CostParams) -> np.ndarray:
@@ -72,6 +91,19 @@ def modeled(x: np.ndarray, params: S.CostParams) -> Dict[str, float]:
     return dict(gpu_us=t, makespan_us=max(t), rank_us=params.gpu_time(x.reshape(-1)))
 
 
+def previous_window_counts(seed: int, T: int, local: Sequence[int]) -> List[int]:
+    """Counts of the window before the batch, the way the off-path thread sees them: another routed batch of
+    the same popularity (seed + 1000) has gone through the cumulative counter, which wrapped on the way."""
+    prev = W.config3("uniform", seed=seed + 1000, T=T)
+    live = prev.topk_ids[:prev.n_valid].reshape(-1)
+    counts = np.bincount(live, minlength=prev.E).astype(np.uint64)
+    snap0 = np.full(prev.E, 2 ** 32 - 7, np.uint64)                       # the counter just before it wraps
+    snap1 = ((snap0 + counts) % (1 << 32)).astype(np.uint32)             # what tempo_count_dispatch leaves behind
+    window = C.window_counts(snap1, snap0.astype(np.uint32))
+    assert np.array_equal(window.astype(np.uint64), counts)
+    return [int(window[e]) for e in local]
+
+
 def build_cases(params: S.CostParams, seed: int = 2, T: int = 4096, policies: Sequence[str] = POLICIES,
                 with_x: bool = True) -> List[PolicyCase]:
     """Config 3's routed batch under each policy."""
@@ -87,13 +119,19 @@ def build_cases(params: S.CostParams, seed: int = 2, T: int = 4096, policies: Se
     flat = ids.reshape(-1)
     cases = []
     for name in policies:
-        x = shares(name, counts, hot, params)
+        if name == "tempo_fast_stale1":
+            # solved on last window's counts; the published table is stale, the kernel renormalises each row
+            table = shares("tempo_fast", previous_window_counts(seed, T, local), hot, params)
+            x = np.array([renormalised(table[i], counts[i]) if i in hot else [counts[i], 0] for i in range(len(local))],
+                         np.int64)
+        else:
+            table = x = shares(name, counts, hot, params)
         # the rank that holds all 20 slots: column 0 = primary slot, column 1 = replica slot
         rmap, quota = base.replica_map.copy(), np.zeros_like(base.quota)
         for i, e in enumerate(local):
-            quota[e, 0] = x[i, 0]
+            quota[e, 0] = table[i, 0]
             if i in hot:
-                quota[e, 1] = x[i, 1]
+                quota[e, 1] = table[i, 1]
         rank = dataclasses.replace(base, name=f"cfg3-policy-{name}", replica_map=rmap, quota=quota, _wcache={})
         # what each virtual GPU sees after the all-to-all: of expert e's pairs in ascending pair index, the first
         # x[i, 0] stay on A and the rest go to B (the contiguous rank runs of the dispatch rule)
@@ -114,5 +152,6 @@ def build_cases(params: S.CostParams, seed: int = 2, T: int = 4096, policies: Se
             gpus.append(W.Workload(f"cfg3-policy-{name}-gpu{'AB'[g]}", base.T, base.k, base.E, len(slots), 1, base.d,
                                    base.f, base.n_valid, gid.reshape(ids.shape).astype(np.int32), base.topk_w, rm, q,
                                    np.asarray(slots, np.int32), base.x, base.seed, base.weight_seed))
-        cases.append(PolicyCase(name, x, rank, gpus))
+        rank_rows = np.array([x[i, 0] for i in range(len(local))] + [x[i, 1] for i in hot], np.int64)
+        cases.append(PolicyCase(name, x, rank, gpus, rank_rows))
     return cases

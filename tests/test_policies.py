@@ -22,11 +22,16 @@ def test_every_policy_is_feasible_and_the_dispatch_honours_it_exactly(cases):
         wl = c.rank
         d = O.count_dispatch(wl.topk_ids, wl.n_valid, wl.replica_map, wl.quota, wl.G_max, wl.M_cap)
         assert int(d["status"]) == 0, c.name
-        for e in range(wl.E):
-            for r in range(wl.R_max):
-                s = int(wl.replica_map[e, r])
-                if s >= 0:
-                    assert int(d["inst_count"][s]) == int(wl.quota[e, r]), (c.name, e, r)
+        assert np.array_equal(d["inst_count"], c.rank_rows), c.name
+        if c.name != "tempo_fast_stale1":                      # a fresh table is honoured entry by entry
+            for e in range(wl.E):
+                for r in range(wl.R_max):
+                    s = int(wl.replica_map[e, r])
+                    if s >= 0:
+                        assert int(d["inst_count"][s]) == int(wl.quota[e, r]), (c.name, e, r)
+        else:                                                   # a stale one is renormalised: the rows still add up
+            assert not np.array_equal(wl.quota.sum(1)[wl.replica_map[:, 0] >= 0],
+                                      np.bincount(wl.topk_ids.reshape(-1), minlength=wl.E)[wl.replica_map[:, 0] >= 0])
         assert int(d["inst_count"][:16].sum()) == int(c.x[:, 0].sum())
         assert int(d["inst_count"][16:].sum()) == int(c.x[:, 1].sum())
 
@@ -56,9 +61,24 @@ def test_the_solvers_table_is_the_best_under_its_own_model(cases):
     m = {c.name: P.modeled(c.x, PARAMS) for c in cases}
     best_proxy = min(m[n]["makespan_us"] for n in ("uniform", "token_balanced", "hot_whole"))
     assert m["tempo_fast"]["makespan_us"] <= best_proxy * (1 + 1e-9)
+    # one window of staleness costs a little and still beats every proxy (the paper's "stale-1" regime)
+    assert m["tempo_fast"]["makespan_us"] <= m["tempo_fast_stale1"]["makespan_us"] <= best_proxy
     # the proxies are not all equal under the model: pricing matters on this batch
     spread = max(v["makespan_us"] for v in m.values()) / m["tempo_fast"]["makespan_us"]
     assert spread > 1.02
     # never worse than the lower bound of Theorem 2's discussion
     counts = [int(v) for v in cases[0].x.sum(1)]
     assert m["tempo_fast"]["makespan_us"] >= S.lower_bound(counts, 2, PARAMS) - 1e-9
+
+
+def test_window_counts_survive_the_wrap_of_the_cumulative_counter():
+    from paper_2608_13057_b200 import costmodel as C
+    prev = np.array([2 ** 32 - 3, 5, 2 ** 31, 0], np.uint32)
+    counts = np.array([10, 0, 2 ** 31 + 7, 123456], np.uint64)
+    now = ((prev.astype(np.uint64) + counts) % (1 << 32)).astype(np.uint32)
+    assert np.array_equal(C.window_counts(now, prev).astype(np.uint64), counts)
+    # the oracle's own counter arithmetic gives the same snapshots
+    ids = np.array([[0], [0], [3]], np.int32)
+    d = O.count_dispatch(ids, 3, np.array([[0], [-1], [-1], [1]], np.int32), np.array([[2], [0], [0], [1]], np.int32), 2,
+                         256, cum_counts=prev)
+    assert C.window_counts(d["cum_counts"], prev).tolist() == [2, 0, 0, 1]
