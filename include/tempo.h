@@ -237,9 +237,9 @@ int tempo_grouped_ffn_gather(const tempo_shape* shape, const void* x_q, const ui
  *   - Limit: M_cap <= 2,097,152 rows (16384 tiles of 128).  A larger M_cap returns
  *     TEMPO_ERR_UNSUPPORTED and launches nothing.
  *   - Allocates nothing, ever.  The first call on each device looks up the array's device address
- *     (cudaGetSymbolAddress, with that device current) and caches it on the host; make that first
- *     call outside any stream capture, and from one thread (two threads racing on a device's first
- *     call both look the address up and store the same value).  Every call enqueues a small cudaMemsetAsync of the counters before the kernel.
+ *     (cudaGetSymbolAddress, with that device current) and caches it on the host (atomically: two
+ *     threads racing on a device's first call both look the address up and store the same value);
+ *     make that first call outside any stream capture.  Every call enqueues a small cudaMemsetAsync of the counters before the kernel.
  *   - All calls on a GPU share the one array: two calls that can overlap on the GPU (different
  *     streams) race on it and give wrong results.  Serialise them, or use tempo_grouped_ffn with a
  *     buffer per stream.

@@ -124,17 +124,19 @@ static int launch_ffn_host(int run_mask, const tempo_shape* s, const void* a_q, 
 constexpr int kStaticMaxTiles = 16384;                       // M_cap <= 128 * 16384 = 2,097,152 rows
 static __device__ __align__(256) int32_t g_ffn_scratch[2 * kStaticMaxTiles];
 constexpr int kMaxDevices = 64;
-static int32_t* g_ffn_scratch_addr[kMaxDevices] = {};
+static std::atomic<int32_t*> g_ffn_scratch_addr[kMaxDevices];   // zero-initialised; every writer stores the same value
 
 static int32_t* static_scratch_for_current_device() {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-  if (g_ffn_scratch_addr[dev] == nullptr) {
+  int32_t* addr = g_ffn_scratch_addr[dev].load(std::memory_order_acquire);
+  if (addr == nullptr) {
     void* ptr = nullptr;
     if (cudaGetSymbolAddress(&ptr, g_ffn_scratch) != cudaSuccess || ptr == nullptr) return nullptr;
-    g_ffn_scratch_addr[dev] = static_cast<int32_t*>(ptr);
+    addr = static_cast<int32_t*>(ptr);
+    g_ffn_scratch_addr[dev].store(addr, std::memory_order_release);
   }
-  return g_ffn_scratch_addr[dev];
+  return addr;
 }
 
 }  // namespace tempo
