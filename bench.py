@@ -848,6 +848,15 @@ def run_policies(args):
                                                      makespan_us=max(meas["gpu_a"]["us"], meas["gpu_b"]["us"]),
                                                      rank_us=meas["rank"]["us"]),
                                     detail=meas))
+    # Does the offline profile transfer to these deployment-like batches?  (Section 5.2: the paper refits the profile on
+    # the records of its microbenchmark and compares it with the offline one.)
+    from paper_2608_13057_b200 import costmodel as C
+    legs = [v for p in out["policies"] for v in p["detail"].values() if v["G_act"] > 0]
+    Gs, Ns, Ts, ts = (np.array([v[k] for v in legs], dtype=np.float64) for k in ("G_act", "N", "tiles", "us"))
+    pred = C.block_time(params.a, params.b, params.c, params.beta, Gs, Ns, params.b2, Ts)
+    out["transfer"] = {"legs": len(legs), "offline_profile_mean_abs_err": float(np.mean(np.abs(pred - ts) / ts)),
+                       "offline_profile_mean_signed_err": float(np.mean((pred - ts) / ts)),
+                       "records": [dict(G=int(g), N=int(n), tiles=int(t_), us=float(u)) for g, n, t_, u in zip(Gs, Ns, Ts, ts)]}
     mk = [p["measured_us"]["makespan_us"] for p in out["policies"]]
     md = [p["modeled_us"]["makespan_us"] for p in out["policies"]]
     out["spread"] = {"measured_worst_over_best": max(mk) / min(mk), "modeled_worst_over_best": max(md) / min(md),
