@@ -140,11 +140,18 @@ __global__ void __launch_bounds__(kDispThreads, 1) count_dispatch_kernel(const D
 #pragma unroll 1
   for (int e = tid; e < E; e += kDispThreads) {
     int n_e = 0, base = 0;
+    // the other CTAs' totals, four remote reads in flight at a time (one at a time costs a distributed-shared-memory
+    // round trip per CTA of the cluster)
 #pragma unroll 1
-    for (int c = 0; c < NC; ++c) {
-      const int v = c == cta ? tot[e] : *cluster.map_shared_rank(tot + e, c);
-      if (c < cta) base += v;
-      n_e += v;
+    for (int c0 = 0; c0 < NC; c0 += 4) {
+      int v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) v[u] = c0 + u < NC ? *cluster.map_shared_rank(tot + e, c0 + u) : 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (c0 + u < cta) base += v[u];
+        n_e += v[u];
+      }
     }
     cbase[e] = base;
     if (cta == 0) {
